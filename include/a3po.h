@@ -1,0 +1,205 @@
+/*
+ * a3po.h — C ABI of the B200 (sm_100a) A-3PO log-prob + loss library.
+ *
+ * The library computes the data-parallel hot path of one A-3PO training step:
+ *   hidden states --LM head + log-softmax + gather--> log pi_theta(a_t|s_t)
+ *   --> A-3PO decoupled clipped loss with the staleness-interpolated proximal anchor
+ *   --> dL/dlogp --> dL/dhidden, dL/dW_lmhead.
+ *
+ * Conventions for every entry point (unless an argument says otherwise):
+ *   - Pointers are DEVICE pointers owned by the caller.  The library allocates no device
+ *     memory: scratch space is the caller's `ws` buffer (size it with the *_workspace_bytes
+ *     functions; 256-byte aligned).  Contents of `ws` are undefined before and after a call.
+ *   - Work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = legacy default
+ *     stream).  Calls never synchronise the device and are asynchronous w.r.t. the host.
+ *   - Return value: A3PO_OK or a negative a3po_error.  Argument errors are detected on the
+ *     host before anything is launched; nothing is written in that case.
+ *   - Conditions that only the device can see (a target index outside [0,V), a bounded wait
+ *     that ran out) are OR-ed into the optional device word `status` (see A3PO_STATUS_*); the
+ *     caller reads it after its own synchronisation.  An out-of-range target is clamped into
+ *     range, never dereferenced.
+ *   - N is the number of token rows.  Row-major layouts: hidden [N,H], W [V,H] (the LM head
+ *     as stored by the model: one row per vocabulary entry), grad_hidden [N,H], grad_w [V,H].
+ *   - `targets[t]` is the token whose probability is wanted at row t (the caller has already
+ *     applied the next-token shift).
+ *   - N = 0 is valid everywhere and is a no-op that still defines scalar outputs (loss = 0).
+ */
+#ifndef A3PO_H_
+#define A3PO_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  A3PO_OK = 0,
+  A3PO_ERR_INVALID_ARG = -1,  /* NULL where a pointer is required, negative size, eps < 0 ...   */
+  A3PO_ERR_UNSUPPORTED = -2,  /* dtype/shape/alignment the kernels do not handle                */
+  A3PO_ERR_WORKSPACE = -3,    /* ws is NULL, misaligned or smaller than the minimum             */
+  A3PO_ERR_CUDA = -4,         /* a CUDA runtime/driver call or a kernel launch failed           */
+  A3PO_ERR_NO_DEVICE = -5     /* no usable sm_100 device is current                             */
+} a3po_error;
+
+/* Storage type of hidden, W and grad_hidden.  Accumulation is always fp32. */
+typedef enum { A3PO_F32 = 0, A3PO_BF16 = 1 } a3po_dtype;
+
+/* Bits of the optional device status word. */
+#define A3PO_STATUS_TARGET_OUT_OF_RANGE 1u /* some targets[t] was outside [0,V) and was clamped */
+#define A3PO_STATUS_WAIT_TIMEOUT 2u        /* a bounded pipeline wait expired; results invalid  */
+
+/* Side outputs of the loss forward: the paper's per-step stability diagnostics
+ * (importance-weight max/min, Fig. 5; number of clipped tokens, Fig. 6). */
+typedef struct {
+  int64_t n_valid;   /* M = number of tokens with mask != 0                                     */
+  int64_t n_clipped; /* valid tokens whose clipped term is the strict minimum (zero gradient)   */
+  float iw_max;      /* max over valid tokens of pi_prox/pi_behav (0 if M == 0)                 */
+  float iw_min;      /* min over valid tokens of pi_prox/pi_behav (0 if M == 0)                 */
+} a3po_stats;
+
+const char* a3po_status_string(int code);
+
+/* Library/ABI version: major*1000 + minor. */
+int a3po_version(void);
+
+/* --------------------------------------------------------------------------------------------
+ * Policy forward, last stage (Sec. 2.2 "forward pass through the model"; Sec. 3: the engines
+ * exchange token log-probabilities; Sec. 4.1: sampling temperature 1.0 => inv_temperature 1).
+ *
+ *   z[t,v]  = inv_temperature * sum_k hidden[t,k] * W[v,k]
+ *   lse[t]  = log sum_v exp(z[t,v])
+ *   logp[t] = z[t, targets[t]] - lse[t]
+ *
+ * The [N,V] logits are never written to memory: the contraction is fused with an online,
+ * vocabulary-chunked log-sum-exp and the target gather.
+ *
+ * hidden [N,H], w [V,H]: dtype `dt`, 16-byte aligned, H % 8 == 0 for A3PO_BF16.
+ * targets int32 [N].  row_mask uint8 [N] or NULL: rows with 0 report logp = lse = 0.
+ * logp, lse: fp32 [N] outputs (lse is needed by the backward).
+ * entropy: fp32 [N] or NULL; when given, receives the policy entropy -sum_v p_v log p_v of
+ *          each row (the diagnostic of Fig. 4), computed in the same vocabulary sweep.
+ * ws/ws_bytes: at least a3po_token_logprobs_workspace_bytes(N,H,V,dt,0).
+ * ------------------------------------------------------------------------------------------ */
+size_t a3po_token_logprobs_workspace_bytes(int64_t N, int H, int V, a3po_dtype dt, int is_bwd);
+
+int a3po_token_logprobs_fwd(const void* hidden, const void* w, const int32_t* targets,
+                            const uint8_t* row_mask, int64_t N, int H, int V, a3po_dtype dt,
+                            float inv_temperature, float* logp, float* lse, float* entropy,
+                            void* ws, size_t ws_bytes, uint32_t* status, void* stream);
+
+/* --------------------------------------------------------------------------------------------
+ * Backward of the above (the derivative of log-softmax + gather; no counterpart formula in the
+ * paper, which leaves the backward to autograd):
+ *
+ *   dz[t,v]          = grad_logp[t] * (1[v == targets[t]] - exp(z[t,v] - lse[t])) * inv_temperature
+ *   grad_hidden[t,:] = sum_v dz[t,v] * W[v,:]                      (dtype dt, [N,H], overwritten)
+ *   grad_w[v,:]      = sum_t dz[t,v] * hidden[t,:]                 (fp32 [V,H])
+ *
+ * lse: the forward's output.  grad_logp fp32 [N]: rows with 0 contribute nothing.
+ * accumulate_grad_w != 0 adds into grad_w (gradient accumulation over the mini-batches of a
+ * training step, Sec. 4.1); 0 overwrites it.
+ * dz is materialised only for a chunk of rows at a time inside `ws` (bf16 for A3PO_BF16);
+ * the chunk length adapts to ws_bytes.  a3po_token_logprobs_workspace_bytes(...,1) returns
+ * the size that lets the library use its preferred chunk; the call fails with
+ * A3PO_ERR_WORKSPACE below a3po_token_logprobs_min_workspace_bytes(...).
+ * ------------------------------------------------------------------------------------------ */
+size_t a3po_token_logprobs_min_workspace_bytes(int64_t N, int H, int V, a3po_dtype dt, int is_bwd);
+
+int a3po_token_logprobs_bwd(const void* hidden, const void* w, const int32_t* targets,
+                            const float* lse, const float* grad_logp, int64_t N, int H, int V,
+                            a3po_dtype dt, float inv_temperature, void* grad_hidden,
+                            float* grad_w, int accumulate_grad_w, void* ws, size_t ws_bytes,
+                            uint32_t* status, void* stream);
+
+/* --------------------------------------------------------------------------------------------
+ * A-3PO loss (Eq. 2 with the proximal policy of Eq. 3 and the coefficient of Eq. 4; argument
+ * names follow Listing 1: behav_logp = old_logp, logp = logprobs, versions, current_version).
+ *
+ *   d_t     = current_version - versions[t]            (integer staleness)
+ *   alpha_t = 1/d_t if d_t >= 1 else 1                 (d <= 0 gives 1, as the listing's where)
+ *   lprox_t = alpha_t * behav_logp[t] + (1 - alpha_t) * logp[t]
+ *   iw_t    = exp(lprox_t - behav_logp[t])             importance weight  pi_prox / pi_behav
+ *   r_t     = exp(logp[t] - lprox_t)                   trust-region ratio pi_theta / pi_prox
+ *   obj_t   = iw_t * min(r_t * adv[t], clip(r_t, 1-eps, 1+eps) * adv[t])
+ *   loss    = - sum_t mask[t] * obj_t / max(M, 1),  M = sum_t mask[t]    (masked token mean)
+ *
+ * The kernels evaluate iw and r through the theorem's closed form r = w^alpha
+ * (w = pi_theta/pi_behav), which is the same function with better fp32 conditioning.
+ *
+ * logp, behav_logp, adv: fp32 [N].  mask: uint8 [N] (0 = ignore; ignored tokens may hold any
+ * bit pattern, NaN included: they are selected out, not multiplied).
+ * versions: int32 [N] (one per token) when versions_per_seq == 0; int32 [B] (one per sequence)
+ *   when versions_per_seq != 0, in which case cu_seqlens int32 [B+1] gives each sequence's row
+ *   range [cu_seqlens[b], cu_seqlens[b+1]) with cu_seqlens[0] = 0 and cu_seqlens[B] = N.
+ * clip_eps >= 0.
+ * loss: fp32 device scalar.  stats: device struct or NULL.
+ * The reduction is a fixed two-stage tree: results are bit-identical from run to run.
+ * ws/ws_bytes: at least a3po_loss_workspace_bytes(N).
+ * ------------------------------------------------------------------------------------------ */
+size_t a3po_loss_workspace_bytes(int64_t N);
+
+int a3po_loss_fwd(const float* logp, const float* behav_logp, const int32_t* versions,
+                  int versions_per_seq, const int32_t* cu_seqlens, int B, int32_t current_version,
+                  const float* adv, const uint8_t* mask, int64_t N, float clip_eps, float* loss,
+                  a3po_stats* stats, void* ws, size_t ws_bytes, void* stream);
+
+/* --------------------------------------------------------------------------------------------
+ * dL/dlogp of the loss above.
+ *
+ *   act_t = 1 if r_t*adv_t <= clip(r_t)*adv_t (the unclipped term is the minimum) else 0
+ *   detach_prox != 0 (default reading: the anchor is a constant, like the recomputed anchor of
+ *   Sec. 2.2 which is "frozen"):      grad_logp[t] = -(gl * mask_t / M) * iw_t * adv_t * r_t * act_t
+ *   detach_prox == 0 (differentiate through Eq. 3 too):
+ *       grad_logp[t] = -(gl * mask_t / M) * ((1 - alpha_t) * obj_t + alpha_t * iw_t * adv_t * r_t * act_t)
+ *
+ * grad_loss: fp32 device scalar gl, or NULL for 1.
+ * fwd_stats: the a3po_stats the forward wrote for the same inputs (supplies M), or NULL, in
+ *   which case the mask is counted first (one extra byte per token of traffic).
+ * grad_logp: fp32 [N] output; masked tokens get exactly 0.
+ * ------------------------------------------------------------------------------------------ */
+int a3po_loss_bwd(const float* logp, const float* behav_logp, const int32_t* versions,
+                  int versions_per_seq, const int32_t* cu_seqlens, int B, int32_t current_version,
+                  const float* adv, const uint8_t* mask, int64_t N, float clip_eps,
+                  int detach_prox, const float* grad_loss, const a3po_stats* fwd_stats,
+                  float* grad_logp, void* ws, size_t ws_bytes, void* stream);
+
+/* Forward and backward in one pass over the inputs (mask counted first, then one stream that
+ * reads 17 B/token and writes 4 B/token).  Outputs as in the two calls above; grad_loss = 1. */
+int a3po_loss_fwd_bwd(const float* logp, const float* behav_logp, const int32_t* versions,
+                      int versions_per_seq, const int32_t* cu_seqlens, int B,
+                      int32_t current_version, const float* adv, const uint8_t* mask, int64_t N,
+                      float clip_eps, int detach_prox, float* loss, a3po_stats* stats,
+                      float* grad_logp, void* ws, size_t ws_bytes, void* stream);
+
+/* --------------------------------------------------------------------------------------------
+ * One whole training-step pass with per-step inputs in HOST memory (no counterpart in the
+ * paper; this is the end-to-end form of the four calls above):
+ *   copies hidden, targets, behav_logp, versions, adv, mask host->device, runs
+ *   token_logprobs_fwd -> loss_fwd_bwd -> token_logprobs_bwd, copies loss + stats back.
+ * h_* are host pointers (pinned memory recommended; pageable works but serialises).
+ * d_w, d_grad_w (accumulated into when accumulate_grad_w != 0), d_grad_hidden ([N,H] dt) and
+ * d_stage/d_ws are device buffers.  d_stage needs a3po_train_step_stage_bytes(N,H,dt) bytes and
+ * d_ws a3po_train_step_workspace_bytes(N,H,V,dt).  h_loss (float) and h_stats are host outputs,
+ * valid after the caller synchronises `stream`.
+ * ------------------------------------------------------------------------------------------ */
+size_t a3po_train_step_stage_bytes(int64_t N, int H, a3po_dtype dt);
+size_t a3po_train_step_workspace_bytes(int64_t N, int H, int V, a3po_dtype dt);
+
+int a3po_train_step_host(const void* h_hidden, const int32_t* h_targets, const float* h_behav_logp,
+                         const int32_t* h_versions, const float* h_adv, const uint8_t* h_mask,
+                         int64_t N, int H, int V, a3po_dtype dt, int32_t current_version,
+                         float clip_eps, float inv_temperature, const void* d_w, float* d_grad_w,
+                         int accumulate_grad_w, void* d_grad_hidden, void* d_stage,
+                         size_t stage_bytes, void* d_ws, size_t ws_bytes, float* h_loss,
+                         a3po_stats* h_stats, uint32_t* d_status, void* stream);
+
+/* Number of kernels this library has launched in the calling process since load
+ * (monotonic; for launch accounting in benchmarks). */
+int64_t a3po_kernel_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* A3PO_H_ */

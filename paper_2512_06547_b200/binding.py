@@ -1,0 +1,267 @@
+"""ctypes binding of liba3po.so: same names as the C ABI, argument marshalling only.
+
+Tensors are torch tensors used as typed device (or, for the host entry, pinned host) buffers;
+torch does none of the arithmetic.  Every function raises if the compiled library is missing or
+a call returns an error code: there is no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import c_char_p, c_float, c_int, c_int32, c_int64, c_size_t, c_void_p
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "lib", "liba3po.so")
+
+A3PO_F32 = 0
+A3PO_BF16 = 1
+STATUS_TARGET_OUT_OF_RANGE = 1
+STATUS_WAIT_TIMEOUT = 2
+
+
+class A3poStats(ctypes.Structure):
+    _fields_ = [("n_valid", c_int64), ("n_clipped", c_int64), ("iw_max", c_float), ("iw_min", c_float)]
+
+
+class A3poError(RuntimeError):
+    def __init__(self, fn, code, text):
+        super().__init__(f"{fn} failed: {text} (code {code})")
+        self.code = code
+
+
+_SIGNATURES = {
+    "a3po_status_string": (c_char_p, [c_int]),
+    "a3po_version": (c_int, []),
+    "a3po_kernel_launch_count": (c_int64, []),
+    "a3po_token_logprobs_workspace_bytes": (c_size_t, [c_int64, c_int, c_int, c_int, c_int]),
+    "a3po_token_logprobs_min_workspace_bytes": (c_size_t, [c_int64, c_int, c_int, c_int, c_int]),
+    "a3po_loss_workspace_bytes": (c_size_t, [c_int64]),
+    "a3po_train_step_stage_bytes": (c_size_t, [c_int64, c_int, c_int]),
+    "a3po_train_step_workspace_bytes": (c_size_t, [c_int64, c_int, c_int, c_int]),
+    "a3po_token_logprobs_fwd": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_int, c_int, c_int, c_float,
+                                        c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p, c_void_p]),
+    "a3po_token_logprobs_bwd": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_int, c_int, c_int,
+                                        c_float, c_void_p, c_void_p, c_int, c_void_p, c_size_t, c_void_p, c_void_p]),
+    "a3po_loss_fwd": (c_int, [c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_int, c_int32, c_void_p, c_void_p,
+                              c_int64, c_float, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
+    "a3po_loss_bwd": (c_int, [c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_int, c_int32, c_void_p, c_void_p,
+                              c_int64, c_float, c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
+    "a3po_loss_fwd_bwd": (c_int, [c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_int, c_int32, c_void_p, c_void_p,
+                                  c_int64, c_float, c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t,
+                                  c_void_p]),
+    "a3po_train_step_host": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_int, c_int,
+                                     c_int, c_int32, c_float, c_float, c_void_p, c_void_p, c_int, c_void_p, c_void_p,
+                                     c_size_t, c_void_p, c_size_t, c_void_p, c_void_p, c_void_p, c_void_p]),
+}
+
+_lib = None
+
+
+def exported_symbols():
+    """Names every build of the library must export (those declared in include/a3po.h)."""
+    return sorted(_SIGNATURES)
+
+
+def load_library(path: str | None = None):
+    """Load liba3po.so once and attach argument types.  Raises if it has not been built."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    p = path or LIB_PATH
+    if not os.path.exists(p):
+        raise RuntimeError(
+            f"{p} not found: build it with `python -m paper_2512_06547_b200.build` "
+            "(there is no fallback implementation)")
+    lib = ctypes.CDLL(p)
+    for name, (res, args) in _SIGNATURES.items():
+        fn = getattr(lib, name)
+        fn.restype = res
+        fn.argtypes = args
+    if path is None:
+        _lib = lib
+    return lib
+
+
+def _check(fn, code):
+    if code != 0:
+        raise A3poError(fn, code, load_library().a3po_status_string(code).decode())
+
+
+def _ptr(t):
+    return None if t is None else c_void_p(t.data_ptr())
+
+
+def _stream(stream=None):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return c_void_p(s.cuda_stream)
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return A3PO_F32
+    if t.dtype == torch.bfloat16:
+        return A3PO_BF16
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def _want(t, dtype, name, device_type="cuda"):
+    if t is None:
+        return
+    if t.dtype != dtype or not t.is_contiguous() or t.device.type != device_type:
+        raise TypeError(f"{name}: expected contiguous {dtype} tensor on {device_type}, got {t.dtype} on {t.device}")
+
+
+# ------------------------------------------------------------------------------ sizes
+def a3po_version() -> int:
+    return load_library().a3po_version()
+
+
+def a3po_kernel_launch_count() -> int:
+    return load_library().a3po_kernel_launch_count()
+
+
+def a3po_token_logprobs_workspace_bytes(N, H, V, dt, is_bwd) -> int:
+    return load_library().a3po_token_logprobs_workspace_bytes(N, H, V, dt, int(is_bwd))
+
+
+def a3po_token_logprobs_min_workspace_bytes(N, H, V, dt, is_bwd) -> int:
+    return load_library().a3po_token_logprobs_min_workspace_bytes(N, H, V, dt, int(is_bwd))
+
+
+def a3po_loss_workspace_bytes(N) -> int:
+    return load_library().a3po_loss_workspace_bytes(N)
+
+
+def a3po_train_step_stage_bytes(N, H, dt) -> int:
+    return load_library().a3po_train_step_stage_bytes(N, H, dt)
+
+
+def a3po_train_step_workspace_bytes(N, H, V, dt) -> int:
+    return load_library().a3po_train_step_workspace_bytes(N, H, V, dt)
+
+
+def new_workspace(nbytes: int, device="cuda") -> torch.Tensor:
+    """A byte buffer usable as `ws` (torch's CUDA allocations are at least 256-byte aligned)."""
+    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+
+
+# ------------------------------------------------------------------------------ LM head
+def a3po_token_logprobs_fwd(hidden, w, targets, logp, lse, ws, *, row_mask=None, entropy=None,
+                            inv_temperature=1.0, status=None, stream=None):
+    dt = _dtype_code(hidden)
+    _want(hidden, hidden.dtype, "hidden"); _want(w, hidden.dtype, "w")
+    _want(targets, torch.int32, "targets"); _want(row_mask, torch.uint8, "row_mask")
+    _want(logp, torch.float32, "logp"); _want(lse, torch.float32, "lse"); _want(entropy, torch.float32, "entropy")
+    _want(status, torch.int32, "status"); _want(ws, torch.uint8, "ws")
+    n, h = hidden.shape
+    v = w.shape[0]
+    if w.shape[1] != h or targets.numel() != n or logp.numel() != n or lse.numel() != n:
+        raise ValueError("shape mismatch")
+    rc = load_library().a3po_token_logprobs_fwd(_ptr(hidden), _ptr(w), _ptr(targets), _ptr(row_mask), n, h, v, dt,
+                                                float(inv_temperature), _ptr(logp), _ptr(lse), _ptr(entropy),
+                                                _ptr(ws), ws.numel(), _ptr(status), _stream(stream))
+    _check("a3po_token_logprobs_fwd", rc)
+
+
+def a3po_token_logprobs_bwd(hidden, w, targets, lse, grad_logp, grad_hidden, grad_w, ws, *, accumulate_grad_w=False,
+                            inv_temperature=1.0, status=None, stream=None):
+    dt = _dtype_code(hidden)
+    _want(hidden, hidden.dtype, "hidden"); _want(w, hidden.dtype, "w"); _want(grad_hidden, hidden.dtype, "grad_hidden")
+    _want(targets, torch.int32, "targets"); _want(lse, torch.float32, "lse"); _want(grad_logp, torch.float32, "grad_logp")
+    _want(grad_w, torch.float32, "grad_w"); _want(status, torch.int32, "status"); _want(ws, torch.uint8, "ws")
+    n, h = hidden.shape
+    v = w.shape[0]
+    if w.shape[1] != h or grad_hidden.shape != hidden.shape or grad_w.shape != w.shape or grad_logp.numel() != n:
+        raise ValueError("shape mismatch")
+    rc = load_library().a3po_token_logprobs_bwd(_ptr(hidden), _ptr(w), _ptr(targets), _ptr(lse), _ptr(grad_logp), n, h,
+                                                v, dt, float(inv_temperature), _ptr(grad_hidden), _ptr(grad_w),
+                                                int(bool(accumulate_grad_w)), _ptr(ws), ws.numel(), _ptr(status),
+                                                _stream(stream))
+    _check("a3po_token_logprobs_bwd", rc)
+
+
+# ------------------------------------------------------------------------------ loss
+def _loss_common(logp, behav_logp, versions, adv, mask, cu_seqlens):
+    _want(logp, torch.float32, "logp"); _want(behav_logp, torch.float32, "behav_logp")
+    _want(versions, torch.int32, "versions"); _want(adv, torch.float32, "adv"); _want(mask, torch.uint8, "mask")
+    _want(cu_seqlens, torch.int32, "cu_seqlens")
+    n = logp.numel()
+    if behav_logp.numel() != n or adv.numel() != n or mask.numel() != n:
+        raise ValueError("shape mismatch")
+    per_seq = cu_seqlens is not None
+    b = cu_seqlens.numel() - 1 if per_seq else 0
+    if per_seq and versions.numel() != b:
+        raise ValueError("versions must have one entry per sequence when cu_seqlens is given")
+    if not per_seq and versions.numel() != n:
+        raise ValueError("versions must have one entry per token")
+    return n, int(per_seq), b
+
+
+def new_stats(device="cuda") -> torch.Tensor:
+    """Device storage for one a3po_stats struct (24 bytes)."""
+    return torch.zeros(ctypes.sizeof(A3poStats), dtype=torch.uint8, device=device)
+
+
+def read_stats(stats: torch.Tensor) -> dict:
+    raw = bytes(stats.cpu().numpy().tobytes())
+    s = A3poStats.from_buffer_copy(raw)
+    return dict(n_valid=s.n_valid, n_clipped=s.n_clipped, iw_max=s.iw_max, iw_min=s.iw_min)
+
+
+def a3po_loss_fwd(logp, behav_logp, versions, current_version, adv, mask, clip_eps, loss, ws, *, stats=None,
+                  cu_seqlens=None, stream=None):
+    n, per_seq, b = _loss_common(logp, behav_logp, versions, adv, mask, cu_seqlens)
+    _want(loss, torch.float32, "loss"); _want(stats, torch.uint8, "stats"); _want(ws, torch.uint8, "ws")
+    rc = load_library().a3po_loss_fwd(_ptr(logp), _ptr(behav_logp), _ptr(versions), per_seq, _ptr(cu_seqlens), b,
+                                      int(current_version), _ptr(adv), _ptr(mask), n, float(clip_eps), _ptr(loss),
+                                      _ptr(stats), _ptr(ws), ws.numel(), _stream(stream))
+    _check("a3po_loss_fwd", rc)
+
+
+def a3po_loss_bwd(logp, behav_logp, versions, current_version, adv, mask, clip_eps, grad_logp, ws, *,
+                  detach_prox=True, grad_loss=None, fwd_stats=None, cu_seqlens=None, stream=None):
+    n, per_seq, b = _loss_common(logp, behav_logp, versions, adv, mask, cu_seqlens)
+    _want(grad_logp, torch.float32, "grad_logp"); _want(grad_loss, torch.float32, "grad_loss")
+    _want(fwd_stats, torch.uint8, "fwd_stats"); _want(ws, torch.uint8, "ws")
+    rc = load_library().a3po_loss_bwd(_ptr(logp), _ptr(behav_logp), _ptr(versions), per_seq, _ptr(cu_seqlens), b,
+                                      int(current_version), _ptr(adv), _ptr(mask), n, float(clip_eps),
+                                      int(bool(detach_prox)), _ptr(grad_loss), _ptr(fwd_stats), _ptr(grad_logp),
+                                      _ptr(ws), ws.numel(), _stream(stream))
+    _check("a3po_loss_bwd", rc)
+
+
+def a3po_loss_fwd_bwd(logp, behav_logp, versions, current_version, adv, mask, clip_eps, loss, grad_logp, ws, *,
+                      detach_prox=True, stats=None, cu_seqlens=None, stream=None):
+    n, per_seq, b = _loss_common(logp, behav_logp, versions, adv, mask, cu_seqlens)
+    _want(loss, torch.float32, "loss"); _want(grad_logp, torch.float32, "grad_logp")
+    _want(stats, torch.uint8, "stats"); _want(ws, torch.uint8, "ws")
+    rc = load_library().a3po_loss_fwd_bwd(_ptr(logp), _ptr(behav_logp), _ptr(versions), per_seq, _ptr(cu_seqlens), b,
+                                          int(current_version), _ptr(adv), _ptr(mask), n, float(clip_eps),
+                                          int(bool(detach_prox)), _ptr(loss), _ptr(stats), _ptr(grad_logp), _ptr(ws),
+                                          ws.numel(), _stream(stream))
+    _check("a3po_loss_fwd_bwd", rc)
+
+
+# ------------------------------------------------------------------------------ whole step, host inputs
+def a3po_train_step_host(h_hidden, h_targets, h_behav_logp, h_versions, h_adv, h_mask, current_version, clip_eps,
+                         d_w, d_grad_w, d_grad_hidden, d_stage, d_ws, h_loss, *, h_stats=None, accumulate_grad_w=False,
+                         inv_temperature=1.0, d_status=None, stream=None):
+    dt = _dtype_code(h_hidden)
+    for t, ty, nm in ((h_hidden, h_hidden.dtype, "h_hidden"), (h_targets, torch.int32, "h_targets"),
+                      (h_behav_logp, torch.float32, "h_behav_logp"), (h_versions, torch.int32, "h_versions"),
+                      (h_adv, torch.float32, "h_adv"), (h_mask, torch.uint8, "h_mask"),
+                      (h_loss, torch.float32, "h_loss"), (h_stats, torch.uint8, "h_stats")):
+        _want(t, ty, nm, device_type="cpu")
+    _want(d_w, h_hidden.dtype, "d_w"); _want(d_grad_w, torch.float32, "d_grad_w")
+    _want(d_grad_hidden, h_hidden.dtype, "d_grad_hidden"); _want(d_stage, torch.uint8, "d_stage")
+    _want(d_ws, torch.uint8, "d_ws"); _want(d_status, torch.int32, "d_status")
+    n, h = h_hidden.shape
+    v = d_w.shape[0]
+    rc = load_library().a3po_train_step_host(
+        _ptr(h_hidden), _ptr(h_targets), _ptr(h_behav_logp), _ptr(h_versions), _ptr(h_adv), _ptr(h_mask), n, h, v, dt,
+        int(current_version), float(clip_eps), float(inv_temperature), _ptr(d_w), _ptr(d_grad_w),
+        int(bool(accumulate_grad_w)), _ptr(d_grad_hidden), _ptr(d_stage), d_stage.numel(), _ptr(d_ws), d_ws.numel(),
+        _ptr(h_loss), _ptr(h_stats), _ptr(d_status), _stream(stream))
+    _check("a3po_train_step_host", rc)

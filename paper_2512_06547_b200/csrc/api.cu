@@ -1,0 +1,326 @@
+// C ABI of the LM-head log-prob calls, the whole-step host entry and library-wide helpers.
+
+#include <cstdlib>
+#include <cstring>
+#include <mutex>
+
+#include "a3po_common.cuh"
+#include "lmhead_internal.cuh"
+
+namespace a3po {
+
+std::atomic<long long> g_launches{0};
+
+int sm_count() {
+  static std::mutex mu;
+  static int cached[64];
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
+    cudaGetLastError();
+    return 0;
+  }
+  std::lock_guard<std::mutex> lock(mu);
+  if (cached[dev] == 0) {
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+      cudaGetLastError();
+      return 0;
+    }
+    cached[dev] = sms;
+  }
+  return cached[dev];
+}
+
+namespace {
+
+constexpr int kMergeThreads = 256;
+constexpr int kSimtTile = 64;
+constexpr long long kSimtChunkRows = 4096;
+constexpr long long kTcChunkRows = 16384;
+
+// Combines the per-split online-softmax partials of each row:
+//   M = max_i m_i, S = sum_i s_i exp(m_i - M), lse = M + log S, logp = z_y - lse,
+//   entropy = lse - (sum_i e_i exp(m_i - M)) / S   with e_i = sum_v exp(z_v - m_i) z_v.
+__global__ void __launch_bounds__(kMergeThreads)
+merge_partials_kernel(const SoftmaxPartial* __restrict__ part, const float* __restrict__ part_ent,
+                      const float* __restrict__ zy, const int32_t* __restrict__ targets,
+                      const uint8_t* __restrict__ row_mask, long long n, int v, int splits, float* __restrict__ logp,
+                      float* __restrict__ lse, float* __restrict__ entropy, uint32_t* status) {
+  const long long t = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (t >= n) return;
+  const int y = targets[t];
+  if ((y < 0 || y >= v) && status) atomicOr(status, A3PO_STATUS_TARGET_OUT_OF_RANGE);
+  if (row_mask && row_mask[t] == 0) {
+    logp[t] = 0.f;
+    lse[t] = 0.f;
+    if (entropy) entropy[t] = 0.f;
+    return;
+  }
+  float m = -INFINITY;
+  for (int i = 0; i < splits; ++i) m = fmaxf(m, part[static_cast<long long>(i) * n + t].m);
+  float s = 0.f, e = 0.f;
+  for (int i = 0; i < splits; ++i) {
+    const SoftmaxPartial q = part[static_cast<long long>(i) * n + t];
+    const float scale = expf(q.m - m);
+    s = fmaf(q.s, scale, s);
+    if (entropy) e = fmaf(part_ent[static_cast<long long>(i) * n + t], scale, e);
+  }
+  const float l = m + logf(s);
+  lse[t] = l;
+  logp[t] = zy[t] - l;
+  if (entropy) entropy[t] = l - e / s;
+}
+
+int simt_fwd_splits(long long n, int v) {
+  const long long row_tiles = (n + kSimtTile - 1) / kSimtTile;
+  const int n_tiles = (v + kSimtTile - 1) / kSimtTile;
+  long long s = row_tiles > 0 ? (148 * 4 + row_tiles - 1) / row_tiles : 1;
+  if (s > n_tiles) s = n_tiles;
+  if (s > 64) s = 64;
+  if (s < 1) s = 1;
+  return static_cast<int>(s);
+}
+
+size_t fwd_ws_for(long long n, int splits) {
+  const size_t rows = static_cast<size_t>(n > 0 ? n : 0);
+  return round_up(rows * splits * sizeof(SoftmaxPartial), 256) + round_up(rows * splits * sizeof(float), 256) +
+         round_up(rows * sizeof(float), 256) + 256;
+}
+
+bool force_simt() {
+  const char* e = std::getenv("A3PO_FORCE_SIMT");
+  return e && e[0] == '1';
+}
+
+bool use_tc(a3po_dtype dt, const void* hidden, const void* w, long long n, int h, int v) {
+  return dt == A3PO_BF16 && !force_simt() && lmhead_tc_supported(hidden, w, n, h, v);
+}
+
+size_t elt_size(a3po_dtype dt) { return dt == A3PO_F32 ? 4 : 2; }
+
+size_t simt_bwd_ws(long long chunk_rows, int v) {
+  return round_up(static_cast<size_t>(chunk_rows) * v * sizeof(float), 256) + 256;
+}
+
+long long clamp_chunk(long long want, long long n, long long quantum) {
+  long long c = want;
+  const long long n_up = (n + quantum - 1) / quantum * quantum;
+  if (c > n_up) c = n_up;
+  if (c < quantum) c = quantum;
+  return c;
+}
+
+int check_lmhead_args(const void* hidden, const void* w, const int32_t* targets, long long n, int h, int v,
+                      a3po_dtype dt, float inv_t) {
+  if (n < 0 || h <= 0 || v <= 0 || !(inv_t > 0.f)) return A3PO_ERR_INVALID_ARG;
+  if (dt != A3PO_F32 && dt != A3PO_BF16) return A3PO_ERR_UNSUPPORTED;
+  if (!w || (n > 0 && (!hidden || !targets))) return A3PO_ERR_INVALID_ARG;
+  if (!aligned_to(hidden, 16) || !aligned_to(w, 16) || !aligned_to(targets, 4)) return A3PO_ERR_UNSUPPORTED;
+  if (sm_count() <= 0) return A3PO_ERR_NO_DEVICE;
+  return A3PO_OK;
+}
+
+}  // namespace
+}  // namespace a3po
+
+using namespace a3po;
+
+extern "C" {
+
+const char* a3po_status_string(int code) {
+  switch (code) {
+    case A3PO_OK: return "ok";
+    case A3PO_ERR_INVALID_ARG: return "invalid argument";
+    case A3PO_ERR_UNSUPPORTED: return "unsupported dtype, shape or alignment";
+    case A3PO_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case A3PO_ERR_CUDA: return "CUDA call or kernel launch failed";
+    case A3PO_ERR_NO_DEVICE: return "no usable CUDA device is current";
+    default: return "unknown a3po status";
+  }
+}
+
+int a3po_version(void) { return 1000; }
+
+int64_t a3po_kernel_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+size_t a3po_token_logprobs_min_workspace_bytes(int64_t N, int H, int V, a3po_dtype dt, int is_bwd) {
+  if (N < 0 || H <= 0 || V <= 0) return 0;
+  if (!is_bwd) {
+    size_t a = fwd_ws_for(N, simt_fwd_splits(N, V));
+    if (dt == A3PO_BF16) {
+      const size_t b = fwd_ws_for(N, lmhead_tc_fwd_splits(N, V));
+      if (b > a) a = b;
+    }
+    return a;
+  }
+  size_t a = simt_bwd_ws(kSimtTile, V);
+  if (dt == A3PO_BF16) {
+    const size_t b = lmhead_tc_bwd_ws_bytes(128, N, H, V);
+    if (b > a) a = b;
+  }
+  return a;
+}
+
+size_t a3po_token_logprobs_workspace_bytes(int64_t N, int H, int V, a3po_dtype dt, int is_bwd) {
+  if (N < 0 || H <= 0 || V <= 0) return 0;
+  if (!is_bwd) return a3po_token_logprobs_min_workspace_bytes(N, H, V, dt, 0);
+  size_t a = simt_bwd_ws(clamp_chunk(kSimtChunkRows, N, kSimtTile), V);
+  if (dt == A3PO_BF16) {
+    const size_t b = lmhead_tc_bwd_ws_bytes(clamp_chunk(kTcChunkRows, N, 128), N, H, V);
+    if (b > a) a = b;
+  }
+  return a;
+}
+
+int a3po_token_logprobs_fwd(const void* hidden, const void* w, const int32_t* targets, const uint8_t* row_mask,
+                            int64_t N, int H, int V, a3po_dtype dt, float inv_temperature, float* logp, float* lse,
+                            float* entropy, void* ws, size_t ws_bytes, uint32_t* status, void* stream_) {
+  A3PO_RETURN_IF(check_lmhead_args(hidden, w, targets, N, H, V, dt, inv_temperature));
+  if (N > 0 && (!logp || !lse)) return A3PO_ERR_INVALID_ARG;
+  if (N == 0) return A3PO_OK;
+  if (!ws || !aligned_to(ws, 256)) return A3PO_ERR_WORKSPACE;
+  cudaStream_t stream = as_stream(stream_);
+  const bool tc = use_tc(dt, hidden, w, N, H, V);
+  const int splits = tc ? lmhead_tc_fwd_splits(N, V) : simt_fwd_splits(N, V);
+  if (ws_bytes < fwd_ws_for(N, splits)) return A3PO_ERR_WORKSPACE;
+  Arena arena(ws, ws_bytes);
+  SoftmaxPartial* part = arena.take<SoftmaxPartial>(static_cast<size_t>(N) * splits);
+  float* part_ent = arena.take<float>(static_cast<size_t>(N) * splits);
+  float* zy = arena.take<float>(static_cast<size_t>(N));
+  if (!arena.ok()) return A3PO_ERR_WORKSPACE;
+  if (!entropy) part_ent = nullptr;
+  if (tc) {
+    A3PO_RETURN_IF(lmhead_fwd_tc(hidden, w, targets, N, H, V, inv_temperature, splits, part, part_ent, zy, status,
+                                 stream));
+  } else {
+    A3PO_RETURN_IF(lmhead_fwd_simt(hidden, w, targets, N, H, V, dt, inv_temperature, splits, part, part_ent, zy,
+                                   stream));
+  }
+  const unsigned blocks = static_cast<unsigned>((N + kMergeThreads - 1) / kMergeThreads);
+  merge_partials_kernel<<<blocks, kMergeThreads, 0, stream>>>(part, part_ent, zy, targets, row_mask, N, V, splits,
+                                                              logp, lse, entropy, status);
+  return after_launch();
+}
+
+int a3po_token_logprobs_bwd(const void* hidden, const void* w, const int32_t* targets, const float* lse,
+                            const float* grad_logp, int64_t N, int H, int V, a3po_dtype dt, float inv_temperature,
+                            void* grad_hidden, float* grad_w, int accumulate_grad_w, void* ws, size_t ws_bytes,
+                            uint32_t* status, void* stream_) {
+  A3PO_RETURN_IF(check_lmhead_args(hidden, w, targets, N, H, V, dt, inv_temperature));
+  if (!grad_w || (N > 0 && (!lse || !grad_logp || !grad_hidden))) return A3PO_ERR_INVALID_ARG;
+  if (!aligned_to(grad_hidden, 16) || !aligned_to(grad_w, 16)) return A3PO_ERR_UNSUPPORTED;
+  if (!ws || !aligned_to(ws, 256)) return A3PO_ERR_WORKSPACE;
+  cudaStream_t stream = as_stream(stream_);
+  if (use_tc(dt, hidden, w, N, H, V) && N > 0) {
+    // largest chunk (multiple of 128 rows) whose scratch fits the caller's buffer
+    long long chunk = clamp_chunk(kTcChunkRows, N, 128);
+    while (chunk > 128 && lmhead_tc_bwd_ws_bytes(chunk, N, H, V) > ws_bytes) chunk -= 128;
+    if (lmhead_tc_bwd_ws_bytes(chunk, N, H, V) > ws_bytes) return A3PO_ERR_WORKSPACE;
+    return lmhead_bwd_tc(hidden, w, targets, lse, grad_logp, N, H, V, inv_temperature, grad_hidden, grad_w,
+                         accumulate_grad_w, ws, ws_bytes, chunk, status, stream);
+  }
+  if (ws_bytes < simt_bwd_ws(kSimtTile, V)) return A3PO_ERR_WORKSPACE;
+  long long chunk = clamp_chunk(kSimtChunkRows, N, kSimtTile);
+  const long long fit = static_cast<long long>((ws_bytes - 256) / (sizeof(float) * static_cast<size_t>(V)));
+  if (chunk > fit) chunk = fit / kSimtTile * kSimtTile;
+  if (chunk < kSimtTile) return A3PO_ERR_WORKSPACE;
+  return lmhead_bwd_simt(hidden, w, targets, lse, grad_logp, N, H, V, dt, inv_temperature, grad_hidden, grad_w,
+                         accumulate_grad_w, static_cast<float*>(ws), chunk, stream);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Whole step with per-step inputs in host memory.
+// ------------------------------------------------------------------------------------------------
+namespace {
+struct StageLayout {
+  size_t hidden, targets, behav, versions, adv, mask, logp, lse, grad_logp, loss, stats, total;
+};
+StageLayout stage_layout(long long n, int h, a3po_dtype dt) {
+  StageLayout s;
+  size_t off = 0;
+  const size_t rows = static_cast<size_t>(n > 0 ? n : 0);
+  auto take = [&](size_t bytes) { size_t o = off; off = round_up(off + bytes, 256); return o; };
+  s.hidden = take(rows * h * elt_size(dt));
+  s.targets = take(rows * 4);
+  s.behav = take(rows * 4);
+  s.versions = take(rows * 4);
+  s.adv = take(rows * 4);
+  s.mask = take(rows);
+  s.logp = take(rows * 4);
+  s.lse = take(rows * 4);
+  s.grad_logp = take(rows * 4);
+  s.loss = take(sizeof(float));
+  s.stats = take(sizeof(a3po_stats));
+  s.total = off;
+  return s;
+}
+}  // namespace
+
+size_t a3po_train_step_stage_bytes(int64_t N, int H, a3po_dtype dt) {
+  if (N < 0 || H <= 0) return 0;
+  return stage_layout(N, H, dt).total;
+}
+
+size_t a3po_train_step_workspace_bytes(int64_t N, int H, int V, a3po_dtype dt) {
+  size_t a = a3po_token_logprobs_workspace_bytes(N, H, V, dt, 0);
+  const size_t b = a3po_token_logprobs_workspace_bytes(N, H, V, dt, 1);
+  const size_t c = a3po_loss_workspace_bytes(N);
+  if (b > a) a = b;
+  if (c > a) a = c;
+  return a;
+}
+
+int a3po_train_step_host(const void* h_hidden, const int32_t* h_targets, const float* h_behav_logp,
+                         const int32_t* h_versions, const float* h_adv, const uint8_t* h_mask, int64_t N, int H,
+                         int V, a3po_dtype dt, int32_t current_version, float clip_eps, float inv_temperature,
+                         const void* d_w, float* d_grad_w, int accumulate_grad_w, void* d_grad_hidden, void* d_stage,
+                         size_t stage_bytes, void* d_ws, size_t ws_bytes, float* h_loss, a3po_stats* h_stats,
+                         uint32_t* d_status, void* stream_) {
+  if (N < 0 || H <= 0 || V <= 0) return A3PO_ERR_INVALID_ARG;
+  if (dt != A3PO_F32 && dt != A3PO_BF16) return A3PO_ERR_UNSUPPORTED;
+  if (!h_loss || !d_w || !d_grad_w || !d_stage || !d_ws) return A3PO_ERR_INVALID_ARG;
+  if (N > 0 && (!h_hidden || !h_targets || !h_behav_logp || !h_versions || !h_adv || !h_mask || !d_grad_hidden))
+    return A3PO_ERR_INVALID_ARG;
+  if (!aligned_to(d_stage, 256)) return A3PO_ERR_WORKSPACE;
+  const StageLayout s = stage_layout(N, H, dt);
+  if (stage_bytes < s.total) return A3PO_ERR_WORKSPACE;
+  cudaStream_t stream = as_stream(stream_);
+  char* base = static_cast<char*>(d_stage);
+  const size_t rows = static_cast<size_t>(N);
+  auto h2d = [&](size_t off, const void* src, size_t bytes) -> bool {
+    return bytes == 0 || cudaMemcpyAsync(base + off, src, bytes, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+  };
+  if (!h2d(s.hidden, h_hidden, rows * H * elt_size(dt)) || !h2d(s.targets, h_targets, rows * 4) ||
+      !h2d(s.behav, h_behav_logp, rows * 4) || !h2d(s.versions, h_versions, rows * 4) ||
+      !h2d(s.adv, h_adv, rows * 4) || !h2d(s.mask, h_mask, rows)) {
+    cudaGetLastError();
+    return A3PO_ERR_CUDA;
+  }
+  const void* hidden = base + s.hidden;
+  const int32_t* targets = reinterpret_cast<const int32_t*>(base + s.targets);
+  const float* behav = reinterpret_cast<const float*>(base + s.behav);
+  const int32_t* versions = reinterpret_cast<const int32_t*>(base + s.versions);
+  const float* adv = reinterpret_cast<const float*>(base + s.adv);
+  const uint8_t* mask = reinterpret_cast<const uint8_t*>(base + s.mask);
+  float* logp = reinterpret_cast<float*>(base + s.logp);
+  float* lse = reinterpret_cast<float*>(base + s.lse);
+  float* grad_logp = reinterpret_cast<float*>(base + s.grad_logp);
+  float* loss = reinterpret_cast<float*>(base + s.loss);
+  a3po_stats* stats = reinterpret_cast<a3po_stats*>(base + s.stats);
+
+  A3PO_RETURN_IF(a3po_token_logprobs_fwd(hidden, d_w, targets, mask, N, H, V, dt, inv_temperature, logp, lse,
+                                         nullptr, d_ws, ws_bytes, d_status, stream_));
+  A3PO_RETURN_IF(a3po_loss_fwd_bwd(logp, behav, versions, 0, nullptr, 0, current_version, adv, mask, N, clip_eps, 1,
+                                   loss, stats, grad_logp, d_ws, ws_bytes, stream_));
+  A3PO_RETURN_IF(a3po_token_logprobs_bwd(hidden, d_w, targets, lse, grad_logp, N, H, V, dt, inv_temperature,
+                                         d_grad_hidden, d_grad_w, accumulate_grad_w, d_ws, ws_bytes, d_status,
+                                         stream_));
+  if (cudaMemcpyAsync(h_loss, loss, sizeof(float), cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+      (h_stats && cudaMemcpyAsync(h_stats, stats, sizeof(a3po_stats), cudaMemcpyDeviceToHost, stream) != cudaSuccess)) {
+    cudaGetLastError();
+    return A3PO_ERR_CUDA;
+  }
+  return A3PO_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,384 @@
+// A-3PO decoupled clipped loss: forward, backward and one-pass forward+backward.
+//
+// Eq. 2 (decoupled clipped objective) with the proximal anchor of Eq. 3 and the staleness
+// coefficient of Eq. 4.  The path is a pure HBM stream: 17 bytes read per token (two fp32
+// log-probs, an int32 version, an fp32 advantage, a uint8 mask) and, for the backward, 4 bytes
+// written.  Each thread handles groups of four consecutive tokens with 128-bit loads (32-bit for
+// the mask), two groups in flight per iteration; reductions go thread -> warp shuffle -> block
+// -> per-block partial -> one finalising block, in a fixed order, so results do not change from
+// run to run.
+
+#include "a3po_common.cuh"
+
+namespace a3po {
+namespace {
+
+constexpr int kLossThreads = 256;
+constexpr int kBlocksPerSm = 8;
+constexpr int kMaxLossBlocks = 4096;
+
+struct alignas(16) LossPartial {
+  double sum;
+  long long n_valid;
+  long long n_clipped;
+  float iw_max;
+  float iw_min;
+};
+
+struct LossArgs {
+  const float* logp;
+  const float* behav;
+  const int32_t* versions;  // per token
+  const float* adv;
+  const uint8_t* mask;
+  long long n;
+  int32_t current_version;
+  float lo;  // 1 - eps
+  float hi;  // 1 + eps
+  int detach;
+  const float* grad_loss;        // device scalar or null
+  const long long* n_valid_ptr;  // device: M, for the backward coefficient
+  float* grad_logp;
+};
+
+enum : int { kFwd = 0, kBwd = 1, kFwdBwd = 2 };
+
+struct Acc {
+  double sum = 0.0;
+  int n_valid = 0;
+  int n_clipped = 0;
+  float iw_max = 0.f;      // valid tokens have iw > 0
+  float iw_min = 3.4e38f;
+};
+
+// One token of Eq. 2-4.  iw and r are evaluated through the closed form of the theorem
+// (r = w^alpha, iw = w^(1-alpha), w = exp(l_theta - l_behav)): the same function as the literal
+// interpolation of Eq. 3 but conditioned on the small difference of the two log-probs.
+template <int MODE>
+__device__ __forceinline__ void token(float lt, float lb, int ver, float a, bool valid,
+                                      const LossArgs& p, float coef, float& fsum, Acc& acc,
+                                      float& grad) {
+  long long d = static_cast<long long>(p.current_version) - static_cast<long long>(ver);
+  float alpha = (d >= 1) ? __frcp_rn(static_cast<float>(d)) : 1.0f;
+  float delta = lt - lb;
+  float ad = alpha * delta;
+  float r = fast_exp2(ad * kLog2e);
+  float iw = fast_exp2((delta - ad) * kLog2e);
+  float s1 = r * a;
+  float s2 = fminf(fmaxf(r, p.lo), p.hi) * a;
+  bool act = s1 <= s2;
+  float obj = iw * fminf(s1, s2);
+  if (MODE != kBwd) {
+    if (valid) {
+      fsum += obj;
+      acc.n_valid += 1;
+      acc.n_clipped += act ? 0 : 1;
+      acc.iw_max = fmaxf(acc.iw_max, iw);
+      acc.iw_min = fminf(acc.iw_min, iw);
+    }
+  }
+  if (MODE != kFwd) {
+    float through = act ? iw * s1 : 0.f;
+    float dobj = p.detach ? through : fmaf(alpha, through - obj, obj);  // (1-a)*obj + a*through
+    grad = valid ? coef * dobj : 0.f;
+  }
+}
+
+template <int MODE>
+__device__ __forceinline__ void group4(long long g, const LossArgs& p, float coef, Acc& acc) {
+  const float4 lt = __ldcs(reinterpret_cast<const float4*>(p.logp) + g);
+  const float4 lb = __ldcs(reinterpret_cast<const float4*>(p.behav) + g);
+  const int4 ver = __ldcs(reinterpret_cast<const int4*>(p.versions) + g);
+  const float4 a = __ldcs(reinterpret_cast<const float4*>(p.adv) + g);
+  const unsigned m = __ldcs(reinterpret_cast<const unsigned*>(p.mask) + g);
+  float fsum = 0.f;
+  float4 gr;
+  token<MODE>(lt.x, lb.x, ver.x, a.x, (m & 0x000000ffu) != 0, p, coef, fsum, acc, gr.x);
+  token<MODE>(lt.y, lb.y, ver.y, a.y, (m & 0x0000ff00u) != 0, p, coef, fsum, acc, gr.y);
+  token<MODE>(lt.z, lb.z, ver.z, a.z, (m & 0x00ff0000u) != 0, p, coef, fsum, acc, gr.z);
+  token<MODE>(lt.w, lb.w, ver.w, a.w, (m & 0xff000000u) != 0, p, coef, fsum, acc, gr.w);
+  if (MODE != kBwd) acc.sum += static_cast<double>(fsum);
+  if (MODE != kFwd) __stcs(reinterpret_cast<float4*>(p.grad_logp) + g, gr);
+}
+
+template <int MODE>
+__device__ __forceinline__ void single(long long t, const LossArgs& p, float coef, Acc& acc) {
+  float fsum = 0.f, gr = 0.f;
+  token<MODE>(p.logp[t], p.behav[t], p.versions[t], p.adv[t], p.mask[t] != 0, p, coef, fsum, acc, gr);
+  if (MODE != kBwd) acc.sum += static_cast<double>(fsum);
+  if (MODE != kFwd) p.grad_logp[t] = gr;
+}
+
+// VEC = true needs 16-byte aligned fp32/int32 arrays and a 4-byte aligned mask.
+template <int MODE, bool VEC>
+__global__ void __launch_bounds__(kLossThreads) loss_kernel(LossArgs p, LossPartial* partials) {
+  float coef = 0.f;
+  if (MODE != kFwd) {
+    long long m = *p.n_valid_ptr;
+    float gl = p.grad_loss ? *p.grad_loss : 1.0f;
+    coef = (m > 0) ? -gl / static_cast<float>(m) : 0.f;
+  }
+  Acc acc;
+  const long long tid = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+  const long long nthreads = static_cast<long long>(gridDim.x) * blockDim.x;
+  if (VEC) {
+    const long long groups = p.n >> 2;
+    long long g = tid;
+    for (; g + nthreads < groups; g += 2 * nthreads) {
+      group4<MODE>(g, p, coef, acc);
+      group4<MODE>(g + nthreads, p, coef, acc);
+    }
+    if (g < groups) group4<MODE>(g, p, coef, acc);
+    const long long t = (groups << 2) + tid;  // ragged tail: at most three tokens
+    if (t < p.n) single<MODE>(t, p, coef, acc);
+  } else {
+    for (long long t = tid; t < p.n; t += nthreads) single<MODE>(t, p, coef, acc);
+  }
+  if (MODE == kBwd) return;
+
+  double sum = warp_sum(acc.sum);
+  long long nv = warp_sum(static_cast<long long>(acc.n_valid));
+  long long nc = warp_sum(static_cast<long long>(acc.n_clipped));
+  float mx = warp_max(acc.iw_max);
+  float mn = warp_min(acc.iw_min);
+  __shared__ LossPartial sh[kLossThreads / kWarp];
+  const int lane = threadIdx.x % kWarp, warp = threadIdx.x / kWarp;
+  if (lane == 0) sh[warp] = LossPartial{sum, nv, nc, mx, mn};
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    LossPartial out = sh[0];
+    for (int w = 1; w < kLossThreads / kWarp; ++w) {
+      out.sum += sh[w].sum;
+      out.n_valid += sh[w].n_valid;
+      out.n_clipped += sh[w].n_clipped;
+      out.iw_max = fmaxf(out.iw_max, sh[w].iw_max);
+      out.iw_min = fminf(out.iw_min, sh[w].iw_min);
+    }
+    partials[blockIdx.x] = out;
+  }
+}
+
+// Sums the per-block partials in a fixed order: loss = -sum / max(M,1), plus the diagnostics.
+__global__ void __launch_bounds__(kLossThreads) loss_finalize_kernel(const LossPartial* partials,
+                                                                    int count, float* loss,
+                                                                    a3po_stats* stats) {
+  __shared__ LossPartial sh[kLossThreads];
+  LossPartial mine{0.0, 0, 0, 0.f, 3.4e38f};
+  for (int i = threadIdx.x; i < count; i += kLossThreads) {
+    const LossPartial q = partials[i];
+    mine.sum += q.sum;
+    mine.n_valid += q.n_valid;
+    mine.n_clipped += q.n_clipped;
+    mine.iw_max = fmaxf(mine.iw_max, q.iw_max);
+    mine.iw_min = fminf(mine.iw_min, q.iw_min);
+  }
+  sh[threadIdx.x] = mine;
+  __syncthreads();
+  for (int s = kLossThreads / 2; s > 0; s >>= 1) {
+    if (threadIdx.x < s) {
+      sh[threadIdx.x].sum += sh[threadIdx.x + s].sum;
+      sh[threadIdx.x].n_valid += sh[threadIdx.x + s].n_valid;
+      sh[threadIdx.x].n_clipped += sh[threadIdx.x + s].n_clipped;
+      sh[threadIdx.x].iw_max = fmaxf(sh[threadIdx.x].iw_max, sh[threadIdx.x + s].iw_max);
+      sh[threadIdx.x].iw_min = fminf(sh[threadIdx.x].iw_min, sh[threadIdx.x + s].iw_min);
+    }
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    const LossPartial t = sh[0];
+    const long long m = t.n_valid;
+    *loss = static_cast<float>(-t.sum / static_cast<double>(m > 0 ? m : 1));
+    if (stats) {
+      stats->n_valid = m;
+      stats->n_clipped = t.n_clipped;
+      stats->iw_max = m > 0 ? t.iw_max : 0.f;
+      stats->iw_min = m > 0 ? t.iw_min : 0.f;
+    }
+  }
+}
+
+// M = number of non-zero mask bytes.  16 mask bytes per load where alignment allows.
+__global__ void __launch_bounds__(kLossThreads) mask_count_kernel(const uint8_t* mask, long long n,
+                                                                 long long* block_counts) {
+  long long count = 0;
+  const long long tid = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+  const long long nthreads = static_cast<long long>(gridDim.x) * blockDim.x;
+  const bool vec = (reinterpret_cast<uintptr_t>(mask) & 15) == 0;
+  long long done = 0;
+  if (vec) {
+    const long long groups = n >> 4;
+    for (long long g = tid; g < groups; g += nthreads) {
+      const uint4 m = __ldg(reinterpret_cast<const uint4*>(mask) + g);
+      count += (__popc(__vcmpne4(m.x, 0u)) + __popc(__vcmpne4(m.y, 0u)) +
+                __popc(__vcmpne4(m.z, 0u)) + __popc(__vcmpne4(m.w, 0u))) >> 3;
+    }
+    done = groups << 4;
+  }
+  for (long long t = done + tid; t < n; t += nthreads) count += mask[t] != 0;
+  count = warp_sum(count);
+  __shared__ long long sh[kLossThreads / kWarp];
+  if (threadIdx.x % kWarp == 0) sh[threadIdx.x / kWarp] = count;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    long long total = 0;
+    for (int w = 0; w < kLossThreads / kWarp; ++w) total += sh[w];
+    block_counts[blockIdx.x] = total;
+  }
+}
+
+__global__ void __launch_bounds__(kLossThreads) mask_count_finalize_kernel(const long long* block_counts,
+                                                                          int count, long long* out) {
+  __shared__ long long sh[kLossThreads];
+  long long mine = 0;
+  for (int i = threadIdx.x; i < count; i += kLossThreads) mine += block_counts[i];
+  sh[threadIdx.x] = mine;
+  __syncthreads();
+  for (int s = kLossThreads / 2; s > 0; s >>= 1) {
+    if (threadIdx.x < s) sh[threadIdx.x] += sh[threadIdx.x + s];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) *out = sh[0];
+}
+
+// versions given per sequence: write the per-token array the streaming kernels read.
+__global__ void __launch_bounds__(kLossThreads) expand_versions_kernel(const int32_t* per_seq,
+                                                                      const int32_t* cu_seqlens, int b,
+                                                                      long long n, int32_t* per_token) {
+  const long long t = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (t >= n) return;
+  int lo = 0, hi = b;  // find the last sequence whose start is <= t
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (static_cast<long long>(cu_seqlens[mid]) <= t) lo = mid; else hi = mid;
+  }
+  per_token[t] = per_seq[lo];
+}
+
+struct LossWs {
+  LossPartial* partials;
+  long long* block_counts;
+  long long* n_valid;
+  int32_t* versions;
+};
+
+size_t loss_ws_bytes(long long n) {
+  return round_up(sizeof(LossPartial) * kMaxLossBlocks, 256) + round_up(sizeof(long long) * kMaxLossBlocks, 256) +
+         256 + round_up(sizeof(int32_t) * static_cast<size_t>(n > 0 ? n : 0), 256) + 256;
+}
+
+int grid_for(long long n_items) {
+  long long want = (n_items + kLossThreads - 1) / kLossThreads;
+  long long cap = static_cast<long long>(sm_count()) * kBlocksPerSm;
+  if (cap > kMaxLossBlocks) cap = kMaxLossBlocks;
+  if (want > cap) want = cap;
+  if (want < 1) want = 1;
+  return static_cast<int>(want);
+}
+
+int run_loss(int mode, const float* logp, const float* behav, const int32_t* versions, int versions_per_seq,
+             const int32_t* cu_seqlens, int b, int32_t current_version, const float* adv, const uint8_t* mask,
+             long long n, float clip_eps, int detach, const float* grad_loss, const a3po_stats* fwd_stats,
+             float* loss, a3po_stats* stats, float* grad_logp, void* ws, size_t ws_bytes, void* stream_) {
+  if (n < 0 || !(clip_eps >= 0.f)) return A3PO_ERR_INVALID_ARG;
+  if (n > 0 && (!logp || !behav || !versions || !adv || !mask)) return A3PO_ERR_INVALID_ARG;
+  if (mode != kBwd && !loss) return A3PO_ERR_INVALID_ARG;
+  if (mode != kFwd && n > 0 && !grad_logp) return A3PO_ERR_INVALID_ARG;
+  if (versions_per_seq && n > 0 && (!cu_seqlens || b <= 0)) return A3PO_ERR_INVALID_ARG;
+  if (!ws || !aligned_to(ws, 256) || ws_bytes < loss_ws_bytes(n)) return A3PO_ERR_WORKSPACE;
+  if (!aligned_to(logp, 4) || !aligned_to(behav, 4) || !aligned_to(versions, 4) || !aligned_to(adv, 4) ||
+      !aligned_to(grad_logp, 4))
+    return A3PO_ERR_UNSUPPORTED;
+  if (sm_count() <= 0) return A3PO_ERR_NO_DEVICE;
+  cudaStream_t stream = as_stream(stream_);
+
+  Arena arena(ws, ws_bytes);
+  LossWs w;
+  w.partials = arena.take<LossPartial>(kMaxLossBlocks);
+  w.block_counts = arena.take<long long>(kMaxLossBlocks);
+  w.n_valid = arena.take<long long>(1);
+  w.versions = arena.take<int32_t>(static_cast<size_t>(n));
+  if (!arena.ok()) return A3PO_ERR_WORKSPACE;
+
+  if (versions_per_seq && n > 0) {
+    const int blocks = static_cast<int>((n + kLossThreads - 1) / kLossThreads);
+    expand_versions_kernel<<<blocks, kLossThreads, 0, stream>>>(versions, cu_seqlens, b, n, w.versions);
+    A3PO_RETURN_IF(after_launch());
+    versions = w.versions;
+  }
+
+  LossArgs p;
+  p.logp = logp; p.behav = behav; p.versions = versions; p.adv = adv; p.mask = mask; p.n = n;
+  p.current_version = current_version;
+  p.lo = 1.0f - clip_eps; p.hi = 1.0f + clip_eps;
+  p.detach = detach;
+  p.grad_loss = grad_loss;
+  p.grad_logp = grad_logp;
+  p.n_valid_ptr = nullptr;
+
+  if (mode != kFwd) {
+    if (fwd_stats) {
+      p.n_valid_ptr = reinterpret_cast<const long long*>(&fwd_stats->n_valid);
+    } else {
+      const int cb = grid_for((n + 15) / 16);
+      mask_count_kernel<<<cb, kLossThreads, 0, stream>>>(mask, n, w.block_counts);
+      A3PO_RETURN_IF(after_launch());
+      mask_count_finalize_kernel<<<1, kLossThreads, 0, stream>>>(w.block_counts, cb, w.n_valid);
+      A3PO_RETURN_IF(after_launch());
+      p.n_valid_ptr = w.n_valid;
+    }
+  }
+
+  const bool vec = aligned_to(logp, 16) && aligned_to(behav, 16) && aligned_to(versions, 16) &&
+                   aligned_to(adv, 16) && aligned_to(mask, 4) && (mode == kFwd || aligned_to(grad_logp, 16));
+  const int blocks = grid_for(vec ? (n + 7) / 8 : n);
+#define A3PO_LAUNCH_LOSS(MODE)                                                                   \
+  do {                                                                                           \
+    if (vec) loss_kernel<MODE, true><<<blocks, kLossThreads, 0, stream>>>(p, w.partials);        \
+    else loss_kernel<MODE, false><<<blocks, kLossThreads, 0, stream>>>(p, w.partials);           \
+  } while (0)
+  if (mode == kFwd) A3PO_LAUNCH_LOSS(kFwd);
+  else if (mode == kBwd) A3PO_LAUNCH_LOSS(kBwd);
+  else A3PO_LAUNCH_LOSS(kFwdBwd);
+#undef A3PO_LAUNCH_LOSS
+  A3PO_RETURN_IF(after_launch());
+  if (mode != kBwd) {
+    loss_finalize_kernel<<<1, kLossThreads, 0, stream>>>(w.partials, blocks, loss, stats);
+    A3PO_RETURN_IF(after_launch());
+  }
+  return A3PO_OK;
+}
+
+}  // namespace
+}  // namespace a3po
+
+extern "C" {
+
+size_t a3po_loss_workspace_bytes(int64_t N) { return a3po::loss_ws_bytes(N); }
+
+int a3po_loss_fwd(const float* logp, const float* behav_logp, const int32_t* versions, int versions_per_seq,
+                  const int32_t* cu_seqlens, int B, int32_t current_version, const float* adv,
+                  const uint8_t* mask, int64_t N, float clip_eps, float* loss, a3po_stats* stats, void* ws,
+                  size_t ws_bytes, void* stream) {
+  return a3po::run_loss(a3po::kFwd, logp, behav_logp, versions, versions_per_seq, cu_seqlens, B, current_version,
+                        adv, mask, N, clip_eps, 1, nullptr, nullptr, loss, stats, nullptr, ws, ws_bytes, stream);
+}
+
+int a3po_loss_bwd(const float* logp, const float* behav_logp, const int32_t* versions, int versions_per_seq,
+                  const int32_t* cu_seqlens, int B, int32_t current_version, const float* adv,
+                  const uint8_t* mask, int64_t N, float clip_eps, int detach_prox, const float* grad_loss,
+                  const a3po_stats* fwd_stats, float* grad_logp, void* ws, size_t ws_bytes, void* stream) {
+  return a3po::run_loss(a3po::kBwd, logp, behav_logp, versions, versions_per_seq, cu_seqlens, B, current_version,
+                        adv, mask, N, clip_eps, detach_prox, grad_loss, fwd_stats, nullptr, nullptr, grad_logp, ws,
+                        ws_bytes, stream);
+}
+
+int a3po_loss_fwd_bwd(const float* logp, const float* behav_logp, const int32_t* versions, int versions_per_seq,
+                      const int32_t* cu_seqlens, int B, int32_t current_version, const float* adv,
+                      const uint8_t* mask, int64_t N, float clip_eps, int detach_prox, float* loss,
+                      a3po_stats* stats, float* grad_logp, void* ws, size_t ws_bytes, void* stream) {
+  return a3po::run_loss(a3po::kFwdBwd, logp, behav_logp, versions, versions_per_seq, cu_seqlens, B,
+                        current_version, adv, mask, N, clip_eps, detach_prox, nullptr, nullptr, loss, stats,
+                        grad_logp, ws, ws_bytes, stream);
+}
+
+}  // extern "C"
