@@ -1,11 +1,595 @@
-// placeholder until the tensor-core kernels land
+// LM-head log-prob forward/backward on the sm_100a tensor cores (bf16 in, fp32 accumulate).
+//
+// One persistent, warp-specialised kernel template does every contraction of the path,
+//     C[M, N] = A[M, K] * B[N, K]^T        (both operands K-major, "TN"),
+// and differs only in its epilogue:
+//   forward      A = hidden, B = W           online (max, sum-exp) per row + target gather
+//   dz           A = hidden, B = W           dz = g (1[v = y] - exp(z - lse)) -> bf16 chunk (+ its transpose)
+//   grad_hidden  A = dz,     B = W^T         bf16 store
+//   grad_w       A = dz^T,   B = hidden^T    fp32 store / accumulate
+//
+// Per CTA (one per SM): warp 0 = TMA producer (one elected lane), warp 1 = tcgen05.mma issuer
+// (one elected lane; it also owns the TMEM allocation), warps 2-5 = epilogue (one TMEM lane
+// quarter each, one accumulator row per thread).  Operand tiles (128 x 64 and 256 x 64 bf16,
+// 128-byte swizzle) move through a 4-stage shared-memory ring guarded by full/empty mbarriers;
+// the 128 x 256 fp32 accumulator is double-buffered in TMEM (2 x 256 columns) so the epilogue
+// of tile i overlaps the MMAs of tile i+1.  Logits never leave TMEM/registers.
+//
+// Every mbarrier wait is bounded; on expiry the CTA raises A3PO_STATUS_WAIT_TIMEOUT in the
+// caller's status word, releases its TMEM and exits.
+
+#include <mutex>
+
+#include "a3po_common.cuh"
 #include "lmhead_internal.cuh"
+#include "sm100_ptx.cuh"
+
 namespace a3po {
-bool lmhead_tc_supported(const void*, const void*, long long, int, int) { return false; }
-int lmhead_tc_fwd_splits(long long, int) { return 1; }
-int lmhead_fwd_tc(const void*, const void*, const int32_t*, long long, int, int, float, int, SoftmaxPartial*, float*,
-                  float*, uint32_t*, cudaStream_t) { return A3PO_ERR_UNSUPPORTED; }
-size_t lmhead_tc_bwd_ws_bytes(long long, long long, int, int) { return 0; }
-int lmhead_bwd_tc(const void*, const void*, const int32_t*, const float*, const float*, long long, int, int, float,
-                  void*, float*, int, void*, size_t, long long, uint32_t*, cudaStream_t) { return A3PO_ERR_UNSUPPORTED; }
+namespace {
+
+using namespace ptx;
+
+constexpr int BM = 128;
+constexpr int BN = 256;
+constexpr int BK = 64;
+constexpr int kStages = 4;
+constexpr int kTcThreads = 192;
+constexpr int kEpiChunk = 32;
+constexpr uint32_t kABytes = BM * BK * 2;
+constexpr uint32_t kBBytes = BN * BK * 2;
+constexpr uint32_t kStageBytes = kABytes + kBBytes;
+constexpr uint32_t kTmemCols = 512;
+constexpr size_t kSmemBytes = 1024 /*alignment slack*/ + kStages * kStageBytes + 256 /*barriers*/;
+constexpr int kGroupM = 16;
+
+// Work decomposition: an item is (row tile, vocabulary split); a split is a contiguous range of
+// column tiles.  Items are ordered so that CTAs running at the same time share row tiles and
+// column tiles through L2: groups of kGroupM row tiles, all splits of a group before the next.
+struct ItemMap {
+  int m_tiles;
+  int n_tiles;
+  int splits;
+  long long items;
+};
+
+struct Item {
+  int m_tile;
+  int split;
+  int n_begin;
+  int n_end;
+};
+
+__device__ __forceinline__ Item decode_item(const ItemMap& im, long long i) {
+  const long long per_group = static_cast<long long>(kGroupM) * im.splits;
+  const int full_groups = im.m_tiles / kGroupM;
+  Item it;
+  if (i < per_group * full_groups) {
+    const int g = static_cast<int>(i / per_group);
+    const int w = static_cast<int>(i % per_group);
+    it.split = w / kGroupM;
+    it.m_tile = g * kGroupM + w % kGroupM;
+  } else {
+    const int rem = im.m_tiles - full_groups * kGroupM;
+    const int w = static_cast<int>(i - per_group * full_groups);
+    it.split = w / rem;
+    it.m_tile = full_groups * kGroupM + w % rem;
+  }
+  it.n_begin = static_cast<int>(static_cast<long long>(it.split) * im.n_tiles / im.splits);
+  it.n_end = static_cast<int>(static_cast<long long>(it.split + 1) * im.n_tiles / im.splits);
+  return it;
 }
+
+__device__ __forceinline__ float bits_to_float(uint32_t u) { return __uint_as_float(u); }
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  __nv_bfloat162 p = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&p);
+}
+
+// ------------------------------------------------------------------------------------ epilogues
+// Each epilogue thread owns one accumulator row (`row` = global row of the A operand).
+// begin(): per-item state; chunk(): 32 consecutive fp32 columns starting at global column `col0`;
+// end(): per-item output.
+
+template <bool ENT>
+struct FwdEpilogue {
+  struct Params {
+    const int32_t* targets;
+    long long n;
+    int v;
+    float scale_log2;  // inv_temperature * log2(e)
+    float inv_t;
+    SoftmaxPartial* part;
+    float* part_ent;
+    float* zy;
+  };
+  float m, s, e;
+  int y;
+  __device__ __forceinline__ void begin(const Params& p, long long row) {
+    m = -INFINITY; s = 0.f; e = 0.f;
+    y = -1;
+    if (row < p.n) y = min(max(p.targets[row], 0), p.v - 1);
+  }
+  __device__ __forceinline__ void chunk(const Params& p, long long row, int col0, uint32_t (&r)[kEpiChunk]) {
+    if (col0 + kEpiChunk > p.v) {  // ragged vocabulary tail: columns past V do not exist
+#pragma unroll
+      for (int j = 0; j < kEpiChunk; ++j)
+        if (col0 + j >= p.v) r[j] = 0xff800000u;  // -inf
+    }
+    float zmax = -INFINITY;
+#pragma unroll
+    for (int j = 0; j < kEpiChunk; ++j) zmax = fmaxf(zmax, bits_to_float(r[j]));
+    const float xm = zmax * p.scale_log2;
+    if (xm > m) {
+      const float f = fast_exp2(m - xm);
+      s *= f;
+      if (ENT) e *= f;
+      m = xm;
+    }
+    float acc = 0.f, ee = 0.f;
+#pragma unroll
+    for (int j = 0; j < kEpiChunk; ++j) {
+      const float z = bits_to_float(r[j]);
+      const float pj = fast_exp2(fmaf(z, p.scale_log2, -m));
+      acc += pj;
+      if (ENT) ee = fmaf(pj, pj > 0.f ? z : 0.f, ee);
+    }
+    s += acc;
+    if (ENT) e = fmaf(ee, p.inv_t, e);
+    if (y >= col0 && y < col0 + kEpiChunk) {
+      float zyv = 0.f;
+#pragma unroll
+      for (int j = 0; j < kEpiChunk; ++j)
+        if (col0 + j == y) zyv = bits_to_float(r[j]);
+      p.zy[row] = zyv * p.inv_t;
+    }
+  }
+  __device__ __forceinline__ void end(const Params& p, long long row, int split) {
+    if (row < p.n) {
+      p.part[static_cast<long long>(split) * p.n + row] = SoftmaxPartial{m * kLn2, s};
+      if (ENT) p.part_ent[static_cast<long long>(split) * p.n + row] = e;
+    }
+  }
+};
+
+struct DzEpilogue {
+  struct Params {
+    const int32_t* targets;   // indexed by global token row
+    const float* lse;
+    const float* grad_logp;
+    long long row_begin;      // first token row of this chunk; A-operand row 0 == row_begin
+    long long row_end;
+    int v;
+    int vpad;                 // row pitch of dz
+    long long tpitch;         // row pitch of dz^T (>= chunk rows)
+    float scale_log2;
+    float inv_t;
+    __nv_bfloat16* dz;        // [chunk rows, vpad]
+    __nv_bfloat16* dzt;       // [v, tpitch]
+  };
+  float g, l2;
+  int y;
+  bool valid;
+  __device__ __forceinline__ void begin(const Params& p, long long row) {
+    const long long t = p.row_begin + row;
+    valid = t < p.row_end;
+    g = 0.f; l2 = INFINITY; y = -1;
+    if (valid) {
+      g = p.grad_logp[t] * p.inv_t;
+      if (g != 0.f) l2 = p.lse[t] * kLog2e;   // g == 0: exp2(-inf) = 0, the row contributes nothing
+      y = min(max(p.targets[t], 0), p.v - 1);
+    }
+  }
+  __device__ __forceinline__ void chunk(const Params& p, long long row, int col0, uint32_t (&r)[kEpiChunk]) {
+    float d[kEpiChunk];
+    const float ng = -g;
+#pragma unroll
+    for (int j = 0; j < kEpiChunk; ++j)
+      d[j] = ng * fast_exp2(fmaf(bits_to_float(r[j]), p.scale_log2, -l2));
+    if (y >= col0 && y < col0 + kEpiChunk) {
+#pragma unroll
+      for (int j = 0; j < kEpiChunk; ++j)
+        if (col0 + j == y) d[j] += g;
+    }
+    if (!valid) return;
+    // row-major copy: 64 contiguous bytes per thread
+    __nv_bfloat16* dst = p.dz + row * p.vpad + col0;
+#pragma unroll
+    for (int q = 0; q < kEpiChunk / 8; ++q) {
+      if (col0 + q * 8 < p.vpad) {
+        uint4 u;
+        u.x = pack_bf16x2(d[q * 8 + 0], d[q * 8 + 1]);
+        u.y = pack_bf16x2(d[q * 8 + 2], d[q * 8 + 3]);
+        u.z = pack_bf16x2(d[q * 8 + 4], d[q * 8 + 5]);
+        u.w = pack_bf16x2(d[q * 8 + 6], d[q * 8 + 7]);
+        *reinterpret_cast<uint4*>(dst + q * 8) = u;
+      }
+    }
+    // transposed copy: the 32 lanes of a warp hold 32 consecutive rows of one column
+#pragma unroll
+    for (int j = 0; j < kEpiChunk; ++j) {
+      const int c = col0 + j;
+      if (c < p.v) p.dzt[static_cast<long long>(c) * p.tpitch + row] = __float2bfloat16_rn(d[j]);
+    }
+  }
+  __device__ __forceinline__ void end(const Params&, long long, int) {}
+};
+
+struct StoreBf16Epilogue {
+  struct Params {
+    __nv_bfloat16* c;
+    long long ldc;
+    long long m_rows;
+    int n_cols;  // multiple of 8
+  };
+  __device__ __forceinline__ void begin(const Params&, long long) {}
+  __device__ __forceinline__ void chunk(const Params& p, long long row, int col0, uint32_t (&r)[kEpiChunk]) {
+    if (row >= p.m_rows) return;
+    __nv_bfloat16* dst = p.c + row * p.ldc + col0;
+#pragma unroll
+    for (int q = 0; q < kEpiChunk / 8; ++q) {
+      if (col0 + q * 8 < p.n_cols) {
+        uint4 u;
+        u.x = pack_bf16x2(bits_to_float(r[q * 8 + 0]), bits_to_float(r[q * 8 + 1]));
+        u.y = pack_bf16x2(bits_to_float(r[q * 8 + 2]), bits_to_float(r[q * 8 + 3]));
+        u.z = pack_bf16x2(bits_to_float(r[q * 8 + 4]), bits_to_float(r[q * 8 + 5]));
+        u.w = pack_bf16x2(bits_to_float(r[q * 8 + 6]), bits_to_float(r[q * 8 + 7]));
+        *reinterpret_cast<uint4*>(dst + q * 8) = u;
+      }
+    }
+  }
+  __device__ __forceinline__ void end(const Params&, long long, int) {}
+};
+
+struct StoreF32Epilogue {
+  struct Params {
+    float* c;
+    long long ldc;
+    long long m_rows;
+    int n_cols;  // multiple of 4
+    int accumulate;
+  };
+  __device__ __forceinline__ void begin(const Params&, long long) {}
+  __device__ __forceinline__ void chunk(const Params& p, long long row, int col0, uint32_t (&r)[kEpiChunk]) {
+    if (row >= p.m_rows) return;
+    float* dst = p.c + row * p.ldc + col0;
+#pragma unroll
+    for (int q = 0; q < kEpiChunk / 4; ++q) {
+      if (col0 + q * 4 < p.n_cols) {
+        float4 o = make_float4(bits_to_float(r[q * 4 + 0]), bits_to_float(r[q * 4 + 1]),
+                               bits_to_float(r[q * 4 + 2]), bits_to_float(r[q * 4 + 3]));
+        if (p.accumulate) {
+          const float4 old = *reinterpret_cast<const float4*>(dst + q * 4);
+          o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
+        }
+        *reinterpret_cast<float4*>(dst + q * 4) = o;
+      }
+    }
+  }
+  __device__ __forceinline__ void end(const Params&, long long, int) {}
+};
+
+// ------------------------------------------------------------------------------------ the kernel
+template <class Epi>
+__global__ void __launch_bounds__(kTcThreads, 1)
+gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, ItemMap im,
+               int k_blocks, typename Epi::Params ep, uint32_t* status) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* smem_a = smem;
+  uint8_t* smem_b = smem + kStages * kABytes;
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + kStages * kStageBytes);
+  uint64_t* empty_bar = full_bar + kStages;
+  uint64_t* tmem_full_bar = empty_bar + kStages;
+  uint64_t* tmem_empty_bar = tmem_full_bar + 2;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tmem_empty_bar + 2);
+  volatile uint32_t* abort_flag = tmem_slot + 1;
+
+  const int warp = threadIdx.x / kWarp;
+  const int lane = threadIdx.x % kWarp;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < kStages; ++i) {
+      mbar_init(&full_bar[i], 1);
+      mbar_init(&empty_bar[i], 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&tmem_full_bar[i], 1);
+      mbar_init(&tmem_empty_bar[i], 4);  // one arrival per epilogue warp
+    }
+    *abort_flag = 0;
+    fence_mbar_init();
+  }
+  if (warp == 0 && lane == 0) {
+    prefetch_tensormap(&map_a);
+    prefetch_tensormap(&map_b);
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_slot, kTmemCols);
+    tmem_relinquish_alloc_permit();
+  }
+  tcgen05_fence_before_sync();
+  __syncthreads();
+  tcgen05_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  bool ok = true;
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (elect_one()) {
+      int stage = 0;
+      uint32_t phase = 0;
+      for (long long i = blockIdx.x; i < im.items && ok; i += gridDim.x) {
+        const Item it = decode_item(im, i);
+        for (int nt = it.n_begin; nt < it.n_end && ok; ++nt) {
+          for (int kb = 0; kb < k_blocks; ++kb) {
+            if (!mbar_wait(&empty_bar[stage], phase ^ 1u, abort_flag)) { ok = false; break; }
+            mbar_arrive_expect_tx(&full_bar[stage], kStageBytes);
+            tma_load_2d(smem_a + stage * kABytes, &map_a, &full_bar[stage], kb * BK, it.m_tile * BM);
+            tma_load_2d(smem_b + stage * kBBytes, &map_b, &full_bar[stage], kb * BK, nt * BN);
+            if (++stage == kStages) { stage = 0; phase ^= 1u; }
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (elect_one()) {
+      constexpr uint32_t idesc = umma_idesc_bf16_f32(BM, BN);
+      int stage = 0;
+      uint32_t phase = 0;
+      int acc = 0;
+      uint32_t acc_phase = 0;
+      for (long long i = blockIdx.x; i < im.items && ok; i += gridDim.x) {
+        const Item it = decode_item(im, i);
+        for (int nt = it.n_begin; nt < it.n_end && ok; ++nt) {
+          if (!mbar_wait(&tmem_empty_bar[acc], acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+          tcgen05_fence_after_sync();
+          const uint32_t tmem_d = tmem_base + static_cast<uint32_t>(acc * BN);
+          for (int kb = 0; kb < k_blocks; ++kb) {
+            if (!mbar_wait(&full_bar[stage], phase, abort_flag)) { ok = false; break; }
+            tcgen05_fence_after_sync();
+            const uint64_t desc_a = umma_desc_k_major_sw128(smem_u32(smem_a + stage * kABytes));
+            const uint64_t desc_b = umma_desc_k_major_sw128(smem_u32(smem_b + stage * kBBytes));
+#pragma unroll
+            for (int k = 0; k < BK / 16; ++k) {
+              // 16 bf16 along K = 32 bytes = 2 descriptor address units inside the swizzled row
+              umma_bf16(tmem_d, desc_a + 2 * k, desc_b + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+            }
+            umma_commit(&empty_bar[stage]);  // stage reusable once these MMAs have read it
+            if (++stage == kStages) { stage = 0; phase ^= 1u; }
+          }
+          if (ok) umma_commit(&tmem_full_bar[acc]);
+          if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue warps
+    const int quarter = warp & 3;  // TMEM lanes this warp may read: 32*quarter .. +31
+    const int row_in_tile = quarter * 32 + lane;
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    Epi epi;
+    for (long long i = blockIdx.x; i < im.items && ok; i += gridDim.x) {
+      const Item it = decode_item(im, i);
+      const long long row = static_cast<long long>(it.m_tile) * BM + row_in_tile;
+      epi.begin(ep, row);
+      for (int nt = it.n_begin; nt < it.n_end && ok; ++nt) {
+        if (!mbar_wait(&tmem_full_bar[acc], acc_phase, abort_flag)) { ok = false; break; }
+        tcgen05_fence_after_sync();
+        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(acc * BN);
+#pragma unroll 1
+        for (int c = 0; c < BN / kEpiChunk; ++c) {
+          uint32_t r[kEpiChunk];
+          tmem_ld_32x32(taddr + static_cast<uint32_t>(c * kEpiChunk), r);
+          tmem_ld_wait();
+          epi.chunk(ep, row, nt * BN + c * kEpiChunk, r);
+        }
+        tcgen05_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&tmem_empty_bar[acc]);
+        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      }
+      if (ok) epi.end(ep, row, it.split);
+    }
+  }
+
+  if (!ok) {
+    *abort_flag = 1;
+    if (status) atomicOr(status, A3PO_STATUS_WAIT_TIMEOUT);
+    __nanosleep(200000);  // let copies / MMAs already in flight drain before TMEM is released
+  }
+  tcgen05_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    tcgen05_fence_after_sync();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// out[c, r] = in[r, c]; in is [rows, cols] with pitch in_pitch, out is [cols, out_pitch].
+__global__ void __launch_bounds__(256) transpose_bf16_kernel(const __nv_bfloat16* __restrict__ in, long long rows,
+                                                            int cols, long long in_pitch,
+                                                            __nv_bfloat16* __restrict__ out, long long out_pitch) {
+  __shared__ __nv_bfloat16 tile[32][34];
+  const int tx = threadIdx.x % 32, ty = threadIdx.x / 32;  // 32 x 8
+  const long long r0 = static_cast<long long>(blockIdx.x) * 32;
+  const int c0 = blockIdx.y * 32;
+  for (int i = ty; i < 32; i += 8) {
+    const long long r = r0 + i;
+    const int c = c0 + tx;
+    tile[i][tx] = (r < rows && c < cols) ? in[r * in_pitch + c] : __float2bfloat16_rn(0.f);
+  }
+  __syncthreads();
+  for (int i = ty; i < 32; i += 8) {
+    const int c = c0 + i;
+    const long long r = r0 + tx;
+    if (c < cols && r < rows) out[static_cast<long long>(c) * out_pitch + r] = tile[tx][i];
+  }
+}
+
+// ------------------------------------------------------------------------------------ host side
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static std::once_flag once;
+  static EncodeTiledFn fn = nullptr;
+  std::call_once(once, [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+    else
+      cudaGetLastError();
+  });
+  return fn;
+}
+
+// 2-D bf16 row-major tensor [outer, inner] with row pitch `pitch` elements; box = [box_outer, 64]
+// with the 128-byte swizzle; out-of-range elements read as zero.
+int make_map(CUtensorMap* map, const void* base, long long inner, long long outer, long long pitch, int box_outer) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return A3PO_ERR_CUDA;
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(inner), static_cast<cuuint64_t>(outer)};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(pitch) * 2};
+  const cuuint32_t box[2] = {static_cast<cuuint32_t>(BK), static_cast<cuuint32_t>(box_outer)};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? A3PO_OK : A3PO_ERR_CUDA;
+}
+
+template <class Epi>
+int launch_gemm(const void* a, long long a_rows, long long a_pitch, const void* b, long long b_rows, long long b_pitch,
+                long long k, int splits, const typename Epi::Params& ep, uint32_t* status, cudaStream_t stream) {
+  CUtensorMap map_a, map_b;
+  A3PO_RETURN_IF(make_map(&map_a, a, k, a_rows, a_pitch, BM));
+  A3PO_RETURN_IF(make_map(&map_b, b, k, b_rows, b_pitch, BN));
+  ItemMap im;
+  im.m_tiles = static_cast<int>((a_rows + BM - 1) / BM);
+  im.n_tiles = static_cast<int>((b_rows + BN - 1) / BN);
+  im.splits = splits > 0 ? splits : im.n_tiles;  // 0: one column tile per item
+  im.items = static_cast<long long>(im.m_tiles) * im.splits;
+  const int k_blocks = static_cast<int>((k + BK - 1) / BK);
+  if (cudaFuncSetAttribute(gemm_tn_kernel<Epi>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           static_cast<int>(kSmemBytes)) != cudaSuccess) {
+    cudaGetLastError();
+    return A3PO_ERR_CUDA;
+  }
+  long long grid = sm_count();
+  if (grid > im.items) grid = im.items;
+  if (grid < 1) return A3PO_OK;
+  gemm_tn_kernel<Epi><<<static_cast<unsigned>(grid), kTcThreads, kSmemBytes, stream>>>(map_a, map_b, im, k_blocks, ep,
+                                                                                      status);
+  return after_launch();
+}
+
+int transpose_bf16(const __nv_bfloat16* in, long long rows, int cols, long long in_pitch, __nv_bfloat16* out,
+                   long long out_pitch, cudaStream_t stream) {
+  if (rows <= 0 || cols <= 0) return A3PO_OK;
+  dim3 grid(static_cast<unsigned>((rows + 31) / 32), static_cast<unsigned>((cols + 31) / 32));
+  transpose_bf16_kernel<<<grid, 256, 0, stream>>>(in, rows, cols, in_pitch, out, out_pitch);
+  return after_launch();
+}
+
+struct BwdWs {
+  size_t wt, ht, dz, dzt, total;
+};
+BwdWs bwd_ws_layout(long long chunk_rows, int h, int v) {
+  const size_t vpad = round_up(static_cast<size_t>(v), 8);
+  BwdWs w;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = round_up(off + bytes, 256); return o; };
+  w.wt = take(static_cast<size_t>(h) * vpad * 2);
+  w.ht = take(static_cast<size_t>(h) * chunk_rows * 2);
+  w.dz = take(static_cast<size_t>(chunk_rows) * vpad * 2);
+  w.dzt = take(static_cast<size_t>(v) * chunk_rows * 2);
+  w.total = off;
+  return w;
+}
+
+}  // namespace
+
+bool lmhead_tc_supported(const void* hidden, const void* w, long long n, int h, int v) {
+  return n > 0 && h >= 8 && (h % 8) == 0 && v >= 1 && aligned_to(hidden, 16) && aligned_to(w, 16) &&
+         n < (1ll << 31) - 256;
+}
+
+// Picks the number of vocabulary splits so that (row tiles x splits) items spread evenly over
+// the SMs (static round-robin) while every item still sweeps several column tiles.
+int lmhead_tc_fwd_splits(long long n, int v) {
+  const long long m_tiles = (n + BM - 1) / BM;
+  const int n_tiles = (v + BN - 1) / BN;
+  if (m_tiles <= 0) return 1;
+  int sms = sm_count();
+  if (sms <= 0) sms = 148;
+  const int s_max = n_tiles < 64 ? n_tiles : 64;
+  int s_min = s_max < 8 ? s_max : 8;  // several splits in flight keep the row-tile working set inside L2
+  int best = s_min;
+  double best_cost = 1e300;
+  for (int s = s_min; s <= s_max; ++s) {
+    const long long items = m_tiles * s;
+    const long long waves = (items + sms - 1) / sms;
+    const long long tiles_per_item = (n_tiles + s - 1) / s;
+    const double cost = static_cast<double>(waves) * (static_cast<double>(tiles_per_item) + 0.5);
+    if (cost < best_cost - 1e-9) { best_cost = cost; best = s; }
+  }
+  return best;
+}
+
+int lmhead_fwd_tc(const void* hidden, const void* w, const int32_t* targets, long long n, int h, int v, float inv_t,
+                  int splits, SoftmaxPartial* part, float* part_ent, float* zy, uint32_t* status,
+                  cudaStream_t stream) {
+  if (part_ent) {
+    FwdEpilogue<true>::Params p{targets, n, v, inv_t * kLog2e, inv_t, part, part_ent, zy};
+    return launch_gemm<FwdEpilogue<true>>(hidden, n, h, w, v, h, h, splits, p, status, stream);
+  }
+  FwdEpilogue<false>::Params p{targets, n, v, inv_t * kLog2e, inv_t, part, nullptr, zy};
+  return launch_gemm<FwdEpilogue<false>>(hidden, n, h, w, v, h, h, splits, p, status, stream);
+}
+
+size_t lmhead_tc_bwd_ws_bytes(long long chunk_rows, long long /*n*/, int h, int v) {
+  return bwd_ws_layout(chunk_rows, h, v).total;
+}
+
+int lmhead_bwd_tc(const void* hidden_, const void* w_, const int32_t* targets, const float* lse,
+                  const float* grad_logp, long long n, int h, int v, float inv_t, void* grad_hidden_, float* grad_w,
+                  int accumulate, void* ws, size_t ws_bytes, long long chunk_rows, uint32_t* status,
+                  cudaStream_t stream) {
+  const __nv_bfloat16* hidden = static_cast<const __nv_bfloat16*>(hidden_);
+  const __nv_bfloat16* w = static_cast<const __nv_bfloat16*>(w_);
+  __nv_bfloat16* grad_hidden = static_cast<__nv_bfloat16*>(grad_hidden_);
+  const BwdWs lay = bwd_ws_layout(chunk_rows, h, v);
+  if (lay.total > ws_bytes) return A3PO_ERR_WORKSPACE;
+  char* base = static_cast<char*>(ws);
+  __nv_bfloat16* wt = reinterpret_cast<__nv_bfloat16*>(base + lay.wt);
+  __nv_bfloat16* ht = reinterpret_cast<__nv_bfloat16*>(base + lay.ht);
+  __nv_bfloat16* dz = reinterpret_cast<__nv_bfloat16*>(base + lay.dz);
+  __nv_bfloat16* dzt = reinterpret_cast<__nv_bfloat16*>(base + lay.dzt);
+  const int vpad = static_cast<int>(round_up(static_cast<size_t>(v), 8));
+
+  A3PO_RETURN_IF(transpose_bf16(w, v, h, h, wt, vpad, stream));  // W^T [h, vpad]
+  for (long long r0 = 0; r0 < n; r0 += chunk_rows) {
+    const long long r1 = (r0 + chunk_rows < n) ? r0 + chunk_rows : n;
+    const long long nc = r1 - r0;
+    const __nv_bfloat16* hid_c = hidden + r0 * h;
+    A3PO_RETURN_IF(transpose_bf16(hid_c, nc, h, h, ht, chunk_rows, stream));  // hidden^T [h, chunk]
+    // dz chunk (and its transpose) from recomputed logits
+    DzEpilogue::Params dp{targets, lse, grad_logp, r0, r1, v, vpad, chunk_rows, inv_t * kLog2e, inv_t, dz, dzt};
+    A3PO_RETURN_IF(launch_gemm<DzEpilogue>(hid_c, nc, h, w, v, h, h, 0, dp, status, stream));
+    // grad_hidden[r0:r1, :] = dz [nc, v] * (W^T [h, v])^T
+    StoreBf16Epilogue::Params hp{grad_hidden + r0 * h, h, nc, h};
+    A3PO_RETURN_IF(launch_gemm<StoreBf16Epilogue>(dz, nc, vpad, wt, h, vpad, v, 0, hp, status, stream));
+    // grad_w (+)= dz^T [v, nc] * (hidden^T [h, nc])^T
+    StoreF32Epilogue::Params wp{grad_w, h, v, h, (accumulate || r0 > 0) ? 1 : 0};
+    A3PO_RETURN_IF(launch_gemm<StoreF32Epilogue>(dzt, v, chunk_rows, ht, h, chunk_rows, nc, 0, wp, status, stream));
+  }
+  return A3PO_OK;
+}
+
+}  // namespace a3po
