@@ -199,6 +199,18 @@ int a3po_train_step_host(const void* h_hidden, const int32_t* h_targets, const f
  * (monotonic; for launch accounting in benchmarks). */
 int64_t a3po_kernel_launch_count(void);
 
+/* --------------------------------------------------------------------------------------------
+ * Optional per-kernel timing (no counterpart in the paper).  While enabled, every kernel the
+ * library launches is bracketed by a pair of CUDA events recorded on the launch stream.
+ * a3po_profile_read waits for the recorded events, returns up to max_entries (kernel id,
+ * milliseconds) pairs in launch order, and clears the record list; a3po_kernel_name maps an id
+ * to a static string.  Host-side state is process-global and mutex-protected.  Leave it off
+ * for production use: each launch costs two extra event records.
+ * ------------------------------------------------------------------------------------------ */
+int a3po_profile_enable(int on);
+int a3po_profile_read(int max_entries, int* kernel_ids, float* milliseconds, int* count);
+const char* a3po_kernel_name(int kernel_id);
+
 #ifdef __cplusplus
 }
 #endif

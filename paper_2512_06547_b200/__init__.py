@@ -14,6 +14,8 @@ from .binding import (  # noqa: F401
     a3po_loss_fwd,
     a3po_loss_fwd_bwd,
     a3po_loss_workspace_bytes,
+    a3po_profile_enable,
+    a3po_profile_read,
     a3po_token_logprobs_bwd,
     a3po_token_logprobs_fwd,
     a3po_token_logprobs_min_workspace_bytes,

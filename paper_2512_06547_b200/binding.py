@@ -35,6 +35,9 @@ _SIGNATURES = {
     "a3po_status_string": (c_char_p, [c_int]),
     "a3po_version": (c_int, []),
     "a3po_kernel_launch_count": (c_int64, []),
+    "a3po_kernel_name": (c_char_p, [c_int]),
+    "a3po_profile_enable": (c_int, [c_int]),
+    "a3po_profile_read": (c_int, [c_int, c_void_p, c_void_p, c_void_p]),
     "a3po_token_logprobs_workspace_bytes": (c_size_t, [c_int64, c_int, c_int, c_int, c_int]),
     "a3po_token_logprobs_min_workspace_bytes": (c_size_t, [c_int64, c_int, c_int, c_int, c_int]),
     "a3po_loss_workspace_bytes": (c_size_t, [c_int64]),
@@ -120,6 +123,20 @@ def a3po_version() -> int:
 
 def a3po_kernel_launch_count() -> int:
     return load_library().a3po_kernel_launch_count()
+
+
+def a3po_profile_enable(on: bool) -> None:
+    _check("a3po_profile_enable", load_library().a3po_profile_enable(int(bool(on))))
+
+
+def a3po_profile_read(max_entries: int = 1 << 16):
+    """Returns [(kernel name, milliseconds), ...] for the launches recorded since the last read."""
+    lib = load_library()
+    ids = (c_int * max_entries)()
+    ms = (c_float * max_entries)()
+    count = c_int(0)
+    _check("a3po_profile_read", lib.a3po_profile_read(max_entries, ids, ms, ctypes.byref(count)))
+    return [(lib.a3po_kernel_name(ids[i]).decode(), float(ms[i])) for i in range(count.value)]
 
 
 def a3po_token_logprobs_workspace_bytes(N, H, V, dt, is_bwd) -> int:

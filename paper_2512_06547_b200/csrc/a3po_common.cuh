@@ -25,6 +25,27 @@ inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 // Number of SMs of the current device (cached per device id).
 int sm_count();
 
+// Kernel identifiers for launch accounting and the optional CUDA-event profile.
+enum KernelId : int {
+  kKLossFwd = 0, kKLossBwd, kKLossFwdBwd, kKLossFinalize, kKMaskCount, kKMaskCountFinalize, kKExpandVersions,
+  kKMergePartials, kKSimtFwd, kKSimtDz, kKSimtGemm, kKTcFwd, kKTcDz, kKTcGradHidden, kKTcGradW, kKTranspose,
+  kKernelIdCount
+};
+
+// When profiling is enabled (a3po_profile_enable), brackets one kernel launch with a pair of CUDA
+// events recorded on the launch stream; otherwise does nothing.
+struct ProfileScope {
+  int slot;
+  cudaStream_t stream;
+  ProfileScope(int kernel_id, cudaStream_t s);
+  ~ProfileScope();
+};
+#define A3PO_LAUNCH(kernel_id, stream, ...)            \
+  do {                                                 \
+    ::a3po::ProfileScope _a3po_scope(kernel_id, stream); \
+    __VA_ARGS__;                                       \
+  } while (0)
+
 // Records one kernel launch and converts a launch error into an a3po_error.
 inline int after_launch() {
   g_launches.fetch_add(1, std::memory_order_relaxed);

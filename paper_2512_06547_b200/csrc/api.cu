@@ -3,6 +3,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <mutex>
+#include <vector>
 
 #include "a3po_common.cuh"
 #include "lmhead_internal.cuh"
@@ -10,6 +11,48 @@
 namespace a3po {
 
 std::atomic<long long> g_launches{0};
+
+// ---- optional CUDA-event profile of every launch -------------------------------------------------
+namespace {
+struct ProfileRecord {
+  int kernel_id;
+  cudaEvent_t start, stop;
+};
+std::mutex g_profile_mu;
+std::atomic<int> g_profile_on{0};
+std::vector<ProfileRecord> g_profile_records;
+std::vector<cudaEvent_t> g_event_pool;
+
+cudaEvent_t take_event() {
+  if (!g_event_pool.empty()) {
+    cudaEvent_t e = g_event_pool.back();
+    g_event_pool.pop_back();
+    return e;
+  }
+  cudaEvent_t e = nullptr;
+  if (cudaEventCreate(&e) != cudaSuccess) {
+    cudaGetLastError();
+    return nullptr;
+  }
+  return e;
+}
+}  // namespace
+
+ProfileScope::ProfileScope(int kernel_id, cudaStream_t s) : slot(-1), stream(s) {
+  if (!g_profile_on.load(std::memory_order_relaxed)) return;
+  std::lock_guard<std::mutex> lock(g_profile_mu);
+  ProfileRecord r{kernel_id, take_event(), take_event()};
+  if (!r.start || !r.stop) return;
+  cudaEventRecord(r.start, stream);
+  g_profile_records.push_back(r);
+  slot = static_cast<int>(g_profile_records.size()) - 1;
+}
+
+ProfileScope::~ProfileScope() {
+  if (slot < 0) return;
+  std::lock_guard<std::mutex> lock(g_profile_mu);
+  if (slot < static_cast<int>(g_profile_records.size())) cudaEventRecord(g_profile_records[slot].stop, stream);
+}
 
 int sm_count() {
   static std::mutex mu;
@@ -143,6 +186,43 @@ int a3po_version(void) { return 1000; }
 
 int64_t a3po_kernel_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
+const char* a3po_kernel_name(int kernel_id) {
+  static const char* names[kKernelIdCount] = {
+      "loss_fwd", "loss_bwd", "loss_fwd_bwd", "loss_finalize", "mask_count", "mask_count_finalize",
+      "expand_versions", "merge_partials", "lmhead_fwd_fp32pipe", "lmhead_dz_fp32pipe", "gemm_fp32pipe",
+      "gemm_tn<fwd_logsoftmax>", "gemm_tn<dz>", "gemm_tn<grad_hidden>", "gemm_tn<grad_w>", "transpose_bf16"};
+  return (kernel_id >= 0 && kernel_id < kKernelIdCount) ? names[kernel_id] : "?";
+}
+
+int a3po_profile_enable(int on) {
+  std::lock_guard<std::mutex> lock(g_profile_mu);
+  g_profile_on.store(on ? 1 : 0);
+  return A3PO_OK;
+}
+
+int a3po_profile_read(int max_entries, int* kernel_ids, float* milliseconds, int* count) {
+  if (!count || max_entries < 0 || (max_entries > 0 && (!kernel_ids || !milliseconds))) return A3PO_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lock(g_profile_mu);
+  int n = 0;
+  int rc = A3PO_OK;
+  for (const ProfileRecord& r : g_profile_records) {
+    float ms = 0.f;
+    if (cudaEventSynchronize(r.stop) != cudaSuccess || cudaEventElapsedTime(&ms, r.start, r.stop) != cudaSuccess) {
+      cudaGetLastError();
+      rc = A3PO_ERR_CUDA;
+    } else if (n < max_entries) {
+      kernel_ids[n] = r.kernel_id;
+      milliseconds[n] = ms;
+      ++n;
+    }
+    g_event_pool.push_back(r.start);
+    g_event_pool.push_back(r.stop);
+  }
+  g_profile_records.clear();
+  *count = n;
+  return rc;
+}
+
 size_t a3po_token_logprobs_min_workspace_bytes(int64_t N, int H, int V, a3po_dtype dt, int is_bwd) {
   if (N < 0 || H <= 0 || V <= 0) return 0;
   if (!is_bwd) {
@@ -197,8 +277,8 @@ int a3po_token_logprobs_fwd(const void* hidden, const void* w, const int32_t* ta
                                    stream));
   }
   const unsigned blocks = static_cast<unsigned>((N + kMergeThreads - 1) / kMergeThreads);
-  merge_partials_kernel<<<blocks, kMergeThreads, 0, stream>>>(part, part_ent, zy, targets, row_mask, N, V, splits,
-                                                              logp, lse, entropy, status);
+  A3PO_LAUNCH(kKMergePartials, stream, (merge_partials_kernel<<<blocks, kMergeThreads, 0, stream>>>(
+                                           part, part_ent, zy, targets, row_mask, N, V, splits, logp, lse, entropy, status)));
   return after_launch();
 }
 

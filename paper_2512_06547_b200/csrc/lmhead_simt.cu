@@ -229,11 +229,11 @@ int fwd_impl(const T* hidden, const T* w, const int32_t* targets, long long n, i
   const int tiles_per_split = (n_tiles + splits - 1) / splits;
   dim3 grid(static_cast<unsigned>((n + kTile - 1) / kTile), static_cast<unsigned>(splits));
   if (part_ent)
-    lmhead_fwd_simt_kernel<T, true><<<grid, kSimtThreads, 0, stream>>>(hidden, w, targets, n, h, v, inv_t,
-                                                                       tiles_per_split, n_tiles, part, part_ent, zy);
+    A3PO_LAUNCH(kKSimtFwd, stream, (lmhead_fwd_simt_kernel<T, true><<<grid, kSimtThreads, 0, stream>>>(
+                                       hidden, w, targets, n, h, v, inv_t, tiles_per_split, n_tiles, part, part_ent, zy)));
   else
-    lmhead_fwd_simt_kernel<T, false><<<grid, kSimtThreads, 0, stream>>>(hidden, w, targets, n, h, v, inv_t,
-                                                                        tiles_per_split, n_tiles, part, nullptr, zy);
+    A3PO_LAUNCH(kKSimtFwd, stream, (lmhead_fwd_simt_kernel<T, false><<<grid, kSimtThreads, 0, stream>>>(
+                                       hidden, w, targets, n, h, v, inv_t, tiles_per_split, n_tiles, part, nullptr, zy)));
   return after_launch();
 }
 
@@ -252,16 +252,17 @@ int bwd_impl(const T* hidden, const T* w, const int32_t* targets, const float* l
     const long long r1 = (r0 + chunk_rows < n) ? r0 + chunk_rows : n;
     const long long nc = r1 - r0;
     const unsigned rt = static_cast<unsigned>((nc + kTile - 1) / kTile);
-    lmhead_dz_simt_kernel<T><<<dim3(rt, vt), kSimtThreads, 0, stream>>>(hidden, w, targets, lse, grad_logp, r0, r1, h,
-                                                                         v, inv_t, ds);
+    A3PO_LAUNCH(kKSimtDz, stream, (lmhead_dz_simt_kernel<T><<<dim3(rt, vt), kSimtThreads, 0, stream>>>(
+                                      hidden, w, targets, lse, grad_logp, r0, r1, h, v, inv_t, ds)));
     A3PO_RETURN_IF(after_launch());
     // grad_hidden[r0:r1, :] = dz @ W
-    gemm_simt_kernel<float, T, T, true><<<dim3(rt, ht), kSimtThreads, 0, stream>>>(
-        ds, v, 1, w, h, grad_hidden + r0 * h, h, nc, h, v, 0);
+    A3PO_LAUNCH(kKSimtGemm, stream, (gemm_simt_kernel<float, T, T, true><<<dim3(rt, ht), kSimtThreads, 0, stream>>>(
+                                        ds, v, 1, w, h, grad_hidden + r0 * h, h, nc, h, v, 0)));
     A3PO_RETURN_IF(after_launch());
     // grad_w (+)= dz^T @ hidden[r0:r1, :]
-    gemm_simt_kernel<float, T, float, false><<<dim3(vt, ht), kSimtThreads, 0, stream>>>(
-        ds, 1, v, hidden + r0 * h, h, grad_w, h, v, h, nc, (accumulate || r0 > 0) ? 1 : 0);
+    A3PO_LAUNCH(kKSimtGemm, stream,
+                (gemm_simt_kernel<float, T, float, false><<<dim3(vt, ht), kSimtThreads, 0, stream>>>(
+                    ds, 1, v, hidden + r0 * h, h, grad_w, h, v, h, nc, (accumulate || r0 > 0) ? 1 : 0)));
     A3PO_RETURN_IF(after_launch());
   }
   return A3PO_OK;

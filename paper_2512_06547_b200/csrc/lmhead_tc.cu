@@ -93,6 +93,7 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 
 template <bool ENT>
 struct FwdEpilogue {
+  static constexpr int kKernelId = kKTcFwd;
   struct Params {
     const int32_t* targets;
     long long n;
@@ -153,6 +154,7 @@ struct FwdEpilogue {
 };
 
 struct DzEpilogue {
+  static constexpr int kKernelId = kKTcDz;
   struct Params {
     const int32_t* targets;   // indexed by global token row
     const float* lse;
@@ -216,6 +218,7 @@ struct DzEpilogue {
 };
 
 struct StoreBf16Epilogue {
+  static constexpr int kKernelId = kKTcGradHidden;
   struct Params {
     __nv_bfloat16* c;
     long long ldc;
@@ -242,6 +245,7 @@ struct StoreBf16Epilogue {
 };
 
 struct StoreF32Epilogue {
+  static constexpr int kKernelId = kKTcGradW;
   struct Params {
     float* c;
     long long ldc;
@@ -484,8 +488,8 @@ int launch_gemm(const void* a, long long a_rows, long long a_pitch, const void* 
   long long grid = sm_count();
   if (grid > im.items) grid = im.items;
   if (grid < 1) return A3PO_OK;
-  gemm_tn_kernel<Epi><<<static_cast<unsigned>(grid), kTcThreads, kSmemBytes, stream>>>(map_a, map_b, im, k_blocks, ep,
-                                                                                      status);
+  A3PO_LAUNCH(Epi::kKernelId, stream, (gemm_tn_kernel<Epi><<<static_cast<unsigned>(grid), kTcThreads, kSmemBytes, stream>>>(
+                                          map_a, map_b, im, k_blocks, ep, status)));
   return after_launch();
 }
 
@@ -493,7 +497,7 @@ int transpose_bf16(const __nv_bfloat16* in, long long rows, int cols, long long 
                    long long out_pitch, cudaStream_t stream) {
   if (rows <= 0 || cols <= 0) return A3PO_OK;
   dim3 grid(static_cast<unsigned>((rows + 31) / 32), static_cast<unsigned>((cols + 31) / 32));
-  transpose_bf16_kernel<<<grid, 256, 0, stream>>>(in, rows, cols, in_pitch, out, out_pitch);
+  A3PO_LAUNCH(kKTranspose, stream, (transpose_bf16_kernel<<<grid, 256, 0, stream>>>(in, rows, cols, in_pitch, out, out_pitch)));
   return after_launch();
 }
 

@@ -301,7 +301,8 @@ int run_loss(int mode, const float* logp, const float* behav, const int32_t* ver
 
   if (versions_per_seq && n > 0) {
     const int blocks = static_cast<int>((n + kLossThreads - 1) / kLossThreads);
-    expand_versions_kernel<<<blocks, kLossThreads, 0, stream>>>(versions, cu_seqlens, b, n, w.versions);
+    A3PO_LAUNCH(kKExpandVersions, stream,
+                expand_versions_kernel<<<blocks, kLossThreads, 0, stream>>>(versions, cu_seqlens, b, n, w.versions));
     A3PO_RETURN_IF(after_launch());
     versions = w.versions;
   }
@@ -320,9 +321,10 @@ int run_loss(int mode, const float* logp, const float* behav, const int32_t* ver
       p.n_valid_ptr = reinterpret_cast<const long long*>(&fwd_stats->n_valid);
     } else {
       const int cb = grid_for((n + 15) / 16);
-      mask_count_kernel<<<cb, kLossThreads, 0, stream>>>(mask, n, w.block_counts);
+      A3PO_LAUNCH(kKMaskCount, stream, mask_count_kernel<<<cb, kLossThreads, 0, stream>>>(mask, n, w.block_counts));
       A3PO_RETURN_IF(after_launch());
-      mask_count_finalize_kernel<<<1, kLossThreads, 0, stream>>>(w.block_counts, cb, w.n_valid);
+      A3PO_LAUNCH(kKMaskCountFinalize, stream,
+                  mask_count_finalize_kernel<<<1, kLossThreads, 0, stream>>>(w.block_counts, cb, w.n_valid));
       A3PO_RETURN_IF(after_launch());
       p.n_valid_ptr = w.n_valid;
     }
@@ -331,18 +333,19 @@ int run_loss(int mode, const float* logp, const float* behav, const int32_t* ver
   const bool vec = aligned_to(logp, 16) && aligned_to(behav, 16) && aligned_to(versions, 16) &&
                    aligned_to(adv, 16) && aligned_to(mask, 4) && (mode == kFwd || aligned_to(grad_logp, 16));
   const int blocks = grid_for(vec ? (n + 7) / 8 : n);
-#define A3PO_LAUNCH_LOSS(MODE)                                                                   \
-  do {                                                                                           \
-    if (vec) loss_kernel<MODE, true><<<blocks, kLossThreads, 0, stream>>>(p, w.partials);        \
-    else loss_kernel<MODE, false><<<blocks, kLossThreads, 0, stream>>>(p, w.partials);           \
+#define A3PO_LAUNCH_LOSS(MODE, KID)                                                                        \
+  do {                                                                                                     \
+    if (vec) A3PO_LAUNCH(KID, stream, (loss_kernel<MODE, true><<<blocks, kLossThreads, 0, stream>>>(p, w.partials)));  \
+    else A3PO_LAUNCH(KID, stream, (loss_kernel<MODE, false><<<blocks, kLossThreads, 0, stream>>>(p, w.partials)));     \
   } while (0)
-  if (mode == kFwd) A3PO_LAUNCH_LOSS(kFwd);
-  else if (mode == kBwd) A3PO_LAUNCH_LOSS(kBwd);
-  else A3PO_LAUNCH_LOSS(kFwdBwd);
+  if (mode == kFwd) A3PO_LAUNCH_LOSS(kFwd, kKLossFwd);
+  else if (mode == kBwd) A3PO_LAUNCH_LOSS(kBwd, kKLossBwd);
+  else A3PO_LAUNCH_LOSS(kFwdBwd, kKLossFwdBwd);
 #undef A3PO_LAUNCH_LOSS
   A3PO_RETURN_IF(after_launch());
   if (mode != kBwd) {
-    loss_finalize_kernel<<<1, kLossThreads, 0, stream>>>(w.partials, blocks, loss, stats);
+    A3PO_LAUNCH(kKLossFinalize, stream,
+                loss_finalize_kernel<<<1, kLossThreads, 0, stream>>>(w.partials, blocks, loss, stats));
     A3PO_RETURN_IF(after_launch());
   }
   return A3PO_OK;
