@@ -1,12 +1,12 @@
 // LM-head log-prob forward/backward on the sm_100a tensor cores (bf16 in, fp32 accumulate).
 //
 // One persistent, warp-specialised kernel template does every contraction of the path,
-//     C[M, N] = A[M, K] * B[N, K]^T        (both operands K-major, "TN"),
+//     C[M, N] = A[M, K] * B[N, K]^T,
 // and differs only in its epilogue:
 //   forward      A = hidden, B = W           online (max, sum-exp) per row + target gather
-//   dz           A = hidden, B = W           dz = g (1[v = y] - exp(z - lse)) -> bf16 chunk (+ its transpose)
-//   grad_hidden  A = dz,     B = W^T         bf16 store
-//   grad_w       A = dz^T,   B = hidden^T    fp32 store / accumulate
+//   dz           A = hidden, B = W           dz = g (1[v = y] - exp(z - lse)) -> bf16 chunk of rows
+//   grad_hidden  A = dz,     B = W^T         bf16 store            (W read in place as an N-major operand)
+//   grad_w       A = dz^T,   B = hidden^T    fp32 store/accumulate (both read in place, M-/N-major)
 //
 // Per CTA (one per SM): warp 0 = TMA producer (one elected lane), warp 1 = tcgen05.mma issuer
 // (one elected lane; it also owns the TMEM allocation), warps 2-5 = epilogue (one TMEM lane
@@ -38,6 +38,7 @@ constexpr int kEpiChunk = 32;
 constexpr uint32_t kABytes = BM * BK * 2;
 constexpr uint32_t kBBytes = BN * BK * 2;
 constexpr uint32_t kStageBytes = kABytes + kBBytes;
+constexpr uint32_t kMnBlockBytes = 64 * BK * 2;  // one 64 (M/N) x 64 (k) box of an MN-major operand
 constexpr uint32_t kTmemCols = 512;
 constexpr size_t kSmemBytes = 1024 /*alignment slack*/ + kStages * kStageBytes + 256 /*barriers*/;
 constexpr int kGroupM = 16;
@@ -163,11 +164,9 @@ struct DzEpilogue {
     long long row_end;
     int v;
     int vpad;                 // row pitch of dz
-    long long tpitch;         // row pitch of dz^T (>= chunk rows)
     float scale_log2;
     float inv_t;
     __nv_bfloat16* dz;        // [chunk rows, vpad]
-    __nv_bfloat16* dzt;       // [v, tpitch]
   };
   float g, l2;
   int y;
@@ -206,12 +205,6 @@ struct DzEpilogue {
         u.w = pack_bf16x2(d[q * 8 + 6], d[q * 8 + 7]);
         *reinterpret_cast<uint4*>(dst + q * 8) = u;
       }
-    }
-    // transposed copy: the 32 lanes of a warp hold 32 consecutive rows of one column
-#pragma unroll
-    for (int j = 0; j < kEpiChunk; ++j) {
-      const int c = col0 + j;
-      if (c < p.v) p.dzt[static_cast<long long>(c) * p.tpitch + row] = __float2bfloat16_rn(d[j]);
     }
   }
   __device__ __forceinline__ void end(const Params&, long long, int) {}
@@ -274,7 +267,10 @@ struct StoreF32Epilogue {
 };
 
 // ------------------------------------------------------------------------------------ the kernel
-template <class Epi>
+// A_MN / B_MN: the operand is read from a tensor whose contiguous index is M (resp. N) instead of
+// K: it arrives as 64 x 64 boxes (64 M/N elements by 64 k) and is fed to the MMA as an MN-major
+// shared-memory matrix, so no transposed copy of the operand ever has to exist in memory.
+template <class Epi, bool A_MN, bool B_MN>
 __global__ void __launch_bounds__(kTcThreads, 1)
 gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, ItemMap im,
                int k_blocks, typename Epi::Params ep, uint32_t* status) {
@@ -329,8 +325,22 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           for (int kb = 0; kb < k_blocks; ++kb) {
             if (!mbar_wait(&empty_bar[stage], phase ^ 1u, abort_flag)) { ok = false; break; }
             mbar_arrive_expect_tx(&full_bar[stage], kStageBytes);
-            tma_load_2d(smem_a + stage * kABytes, &map_a, &full_bar[stage], kb * BK, it.m_tile * BM);
-            tma_load_2d(smem_b + stage * kBBytes, &map_b, &full_bar[stage], kb * BK, nt * BN);
+            uint8_t* sa = smem_a + stage * kABytes;
+            uint8_t* sb = smem_b + stage * kBBytes;
+            if (A_MN) {
+#pragma unroll
+              for (int j = 0; j < BM / 64; ++j)
+                tma_load_2d(sa + j * kMnBlockBytes, &map_a, &full_bar[stage], it.m_tile * BM + j * 64, kb * BK);
+            } else {
+              tma_load_2d(sa, &map_a, &full_bar[stage], kb * BK, it.m_tile * BM);
+            }
+            if (B_MN) {
+#pragma unroll
+              for (int j = 0; j < BN / 64; ++j)
+                tma_load_2d(sb + j * kMnBlockBytes, &map_b, &full_bar[stage], nt * BN + j * 64, kb * BK);
+            } else {
+              tma_load_2d(sb, &map_b, &full_bar[stage], kb * BK, nt * BN);
+            }
             if (++stage == kStages) { stage = 0; phase ^= 1u; }
           }
         }
@@ -339,7 +349,11 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (elect_one()) {
-      constexpr uint32_t idesc = umma_idesc_bf16_f32(BM, BN);
+      constexpr uint32_t idesc = umma_idesc_bf16_f32(BM, BN, A_MN, B_MN);
+      // descriptor start-address step (16-byte units) per UMMA (K = 16): 32 bytes inside the swizzled
+      // row for a K-major tile, two 1024-byte k-group atoms for an MN-major tile
+      constexpr uint32_t a_step = A_MN ? (2 * 1024) >> 4 : 32 >> 4;
+      constexpr uint32_t b_step = B_MN ? (2 * 1024) >> 4 : 32 >> 4;
       int stage = 0;
       uint32_t phase = 0;
       int acc = 0;
@@ -353,13 +367,13 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           for (int kb = 0; kb < k_blocks; ++kb) {
             if (!mbar_wait(&full_bar[stage], phase, abort_flag)) { ok = false; break; }
             tcgen05_fence_after_sync();
-            const uint64_t desc_a = umma_desc_k_major_sw128(smem_u32(smem_a + stage * kABytes));
-            const uint64_t desc_b = umma_desc_k_major_sw128(smem_u32(smem_b + stage * kBBytes));
+            const uint32_t sa = smem_u32(smem_a + stage * kABytes);
+            const uint32_t sb = smem_u32(smem_b + stage * kBBytes);
+            const uint64_t desc_a = A_MN ? umma_desc_mn_major_sw128(sa, kMnBlockBytes) : umma_desc_k_major_sw128(sa);
+            const uint64_t desc_b = B_MN ? umma_desc_mn_major_sw128(sb, kMnBlockBytes) : umma_desc_k_major_sw128(sb);
 #pragma unroll
-            for (int k = 0; k < BK / 16; ++k) {
-              // 16 bf16 along K = 32 bytes = 2 descriptor address units inside the swizzled row
-              umma_bf16(tmem_d, desc_a + 2 * k, desc_b + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
-            }
+            for (int k = 0; k < BK / 16; ++k)
+              umma_bf16(tmem_d, desc_a + a_step * k, desc_b + b_step * k, idesc, (kb | k) != 0 ? 1u : 0u);
             umma_commit(&empty_bar[stage]);  // stage reusable once these MMAs have read it
             if (++stage == kStages) { stage = 0; phase ^= 1u; }
           }
@@ -412,27 +426,6 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   }
 }
 
-// out[c, r] = in[r, c]; in is [rows, cols] with pitch in_pitch, out is [cols, out_pitch].
-__global__ void __launch_bounds__(256) transpose_bf16_kernel(const __nv_bfloat16* __restrict__ in, long long rows,
-                                                            int cols, long long in_pitch,
-                                                            __nv_bfloat16* __restrict__ out, long long out_pitch) {
-  __shared__ __nv_bfloat16 tile[32][34];
-  const int tx = threadIdx.x % 32, ty = threadIdx.x / 32;  // 32 x 8
-  const long long r0 = static_cast<long long>(blockIdx.x) * 32;
-  const int c0 = blockIdx.y * 32;
-  for (int i = ty; i < 32; i += 8) {
-    const long long r = r0 + i;
-    const int c = c0 + tx;
-    tile[i][tx] = (r < rows && c < cols) ? in[r * in_pitch + c] : __float2bfloat16_rn(0.f);
-  }
-  __syncthreads();
-  for (int i = ty; i < 32; i += 8) {
-    const int c = c0 + i;
-    const long long r = r0 + tx;
-    if (c < cols && r < rows) out[static_cast<long long>(c) * out_pitch + r] = tile[tx][i];
-  }
-}
-
 // ------------------------------------------------------------------------------------ host side
 using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -453,68 +446,62 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// 2-D bf16 row-major tensor [outer, inner] with row pitch `pitch` elements; box = [box_outer, 64]
-// with the 128-byte swizzle; out-of-range elements read as zero.
-int make_map(CUtensorMap* map, const void* base, long long inner, long long outer, long long pitch, int box_outer) {
+// One GEMM operand as it lies in memory (bf16, row-major with `pitch` elements per row).
+//   K-major : tensor [mn_extent rows, k_extent cols]   -> boxes of tile_mn rows x 64 k
+//   MN-major: tensor [k_extent rows, mn_extent cols]   -> boxes of 64 k rows x 64 M/N elements
+// Out-of-range elements read as zero, which is what makes ragged M, N and K tails work.
+struct Operand {
+  const void* base;
+  long long mn_extent;
+  long long k_extent;
+  long long pitch;
+};
+
+int make_map(CUtensorMap* map, const Operand& op, bool mn_major, int tile_mn) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return A3PO_ERR_CUDA;
-  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(inner), static_cast<cuuint64_t>(outer)};
-  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(pitch) * 2};
-  const cuuint32_t box[2] = {static_cast<cuuint32_t>(BK), static_cast<cuuint32_t>(box_outer)};
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(mn_major ? op.mn_extent : op.k_extent),
+                              static_cast<cuuint64_t>(mn_major ? op.k_extent : op.mn_extent)};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(op.pitch) * 2};
+  const cuuint32_t box[2] = {64u, static_cast<cuuint32_t>(mn_major ? BK : tile_mn)};
   const cuuint32_t estr[2] = {1, 1};
-  const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(op.base), dims, strides, box,
+                        estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? A3PO_OK : A3PO_ERR_CUDA;
 }
 
-template <class Epi>
-int launch_gemm(const void* a, long long a_rows, long long a_pitch, const void* b, long long b_rows, long long b_pitch,
-                long long k, int splits, const typename Epi::Params& ep, uint32_t* status, cudaStream_t stream) {
+// C[M, N] = sum_k A[m, k] B[n, k];  splits = 0 means one column tile per work item.
+template <class Epi, bool A_MN, bool B_MN>
+int launch_gemm(const Operand& a, const Operand& b, int splits, const typename Epi::Params& ep, uint32_t* status,
+                cudaStream_t stream) {
   CUtensorMap map_a, map_b;
-  A3PO_RETURN_IF(make_map(&map_a, a, k, a_rows, a_pitch, BM));
-  A3PO_RETURN_IF(make_map(&map_b, b, k, b_rows, b_pitch, BN));
+  A3PO_RETURN_IF(make_map(&map_a, a, A_MN, BM));
+  A3PO_RETURN_IF(make_map(&map_b, b, B_MN, BN));
   ItemMap im;
-  im.m_tiles = static_cast<int>((a_rows + BM - 1) / BM);
-  im.n_tiles = static_cast<int>((b_rows + BN - 1) / BN);
-  im.splits = splits > 0 ? splits : im.n_tiles;  // 0: one column tile per item
+  im.m_tiles = static_cast<int>((a.mn_extent + BM - 1) / BM);
+  im.n_tiles = static_cast<int>((b.mn_extent + BN - 1) / BN);
+  im.splits = splits > 0 ? splits : im.n_tiles;
   im.items = static_cast<long long>(im.m_tiles) * im.splits;
-  const int k_blocks = static_cast<int>((k + BK - 1) / BK);
-  if (cudaFuncSetAttribute(gemm_tn_kernel<Epi>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           static_cast<int>(kSmemBytes)) != cudaSuccess) {
+  const int k_blocks = static_cast<int>((a.k_extent + BK - 1) / BK);
+  auto kernel = gemm_tn_kernel<Epi, A_MN, B_MN>;
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemBytes)) !=
+      cudaSuccess) {
     cudaGetLastError();
     return A3PO_ERR_CUDA;
   }
   long long grid = sm_count();
   if (grid > im.items) grid = im.items;
   if (grid < 1) return A3PO_OK;
-  A3PO_LAUNCH(Epi::kKernelId, stream, (gemm_tn_kernel<Epi><<<static_cast<unsigned>(grid), kTcThreads, kSmemBytes, stream>>>(
+  A3PO_LAUNCH(Epi::kKernelId, stream, (kernel<<<static_cast<unsigned>(grid), kTcThreads, kSmemBytes, stream>>>(
                                           map_a, map_b, im, k_blocks, ep, status)));
   return after_launch();
 }
 
-int transpose_bf16(const __nv_bfloat16* in, long long rows, int cols, long long in_pitch, __nv_bfloat16* out,
-                   long long out_pitch, cudaStream_t stream) {
-  if (rows <= 0 || cols <= 0) return A3PO_OK;
-  dim3 grid(static_cast<unsigned>((rows + 31) / 32), static_cast<unsigned>((cols + 31) / 32));
-  A3PO_LAUNCH(kKTranspose, stream, (transpose_bf16_kernel<<<grid, 256, 0, stream>>>(in, rows, cols, in_pitch, out, out_pitch)));
-  return after_launch();
-}
-
-struct BwdWs {
-  size_t wt, ht, dz, dzt, total;
-};
-BwdWs bwd_ws_layout(long long chunk_rows, int h, int v) {
+// Scratch of the backward: one bf16 dz chunk [chunk_rows, vpad].
+size_t bwd_ws_layout(long long chunk_rows, int v) {
   const size_t vpad = round_up(static_cast<size_t>(v), 8);
-  BwdWs w;
-  size_t off = 0;
-  auto take = [&](size_t bytes) { size_t o = off; off = round_up(off + bytes, 256); return o; };
-  w.wt = take(static_cast<size_t>(h) * vpad * 2);
-  w.ht = take(static_cast<size_t>(h) * chunk_rows * 2);
-  w.dz = take(static_cast<size_t>(chunk_rows) * vpad * 2);
-  w.dzt = take(static_cast<size_t>(v) * chunk_rows * 2);
-  w.total = off;
-  return w;
+  return round_up(static_cast<size_t>(chunk_rows) * vpad * 2, 256);
 }
 
 }  // namespace
@@ -549,16 +536,18 @@ int lmhead_tc_fwd_splits(long long n, int v) {
 int lmhead_fwd_tc(const void* hidden, const void* w, const int32_t* targets, long long n, int h, int v, float inv_t,
                   int splits, SoftmaxPartial* part, float* part_ent, float* zy, uint32_t* status,
                   cudaStream_t stream) {
+  const Operand a{hidden, n, h, h};
+  const Operand b{w, v, h, h};
   if (part_ent) {
     FwdEpilogue<true>::Params p{targets, n, v, inv_t * kLog2e, inv_t, part, part_ent, zy};
-    return launch_gemm<FwdEpilogue<true>>(hidden, n, h, w, v, h, h, splits, p, status, stream);
+    return launch_gemm<FwdEpilogue<true>, false, false>(a, b, splits, p, status, stream);
   }
   FwdEpilogue<false>::Params p{targets, n, v, inv_t * kLog2e, inv_t, part, nullptr, zy};
-  return launch_gemm<FwdEpilogue<false>>(hidden, n, h, w, v, h, h, splits, p, status, stream);
+  return launch_gemm<FwdEpilogue<false>, false, false>(a, b, splits, p, status, stream);
 }
 
-size_t lmhead_tc_bwd_ws_bytes(long long chunk_rows, long long /*n*/, int h, int v) {
-  return bwd_ws_layout(chunk_rows, h, v).total;
+size_t lmhead_tc_bwd_ws_bytes(long long chunk_rows, long long /*n*/, int /*h*/, int v) {
+  return bwd_ws_layout(chunk_rows, v);
 }
 
 int lmhead_bwd_tc(const void* hidden_, const void* w_, const int32_t* targets, const float* lse,
@@ -568,30 +557,26 @@ int lmhead_bwd_tc(const void* hidden_, const void* w_, const int32_t* targets, c
   const __nv_bfloat16* hidden = static_cast<const __nv_bfloat16*>(hidden_);
   const __nv_bfloat16* w = static_cast<const __nv_bfloat16*>(w_);
   __nv_bfloat16* grad_hidden = static_cast<__nv_bfloat16*>(grad_hidden_);
-  const BwdWs lay = bwd_ws_layout(chunk_rows, h, v);
-  if (lay.total > ws_bytes) return A3PO_ERR_WORKSPACE;
-  char* base = static_cast<char*>(ws);
-  __nv_bfloat16* wt = reinterpret_cast<__nv_bfloat16*>(base + lay.wt);
-  __nv_bfloat16* ht = reinterpret_cast<__nv_bfloat16*>(base + lay.ht);
-  __nv_bfloat16* dz = reinterpret_cast<__nv_bfloat16*>(base + lay.dz);
-  __nv_bfloat16* dzt = reinterpret_cast<__nv_bfloat16*>(base + lay.dzt);
+  if (bwd_ws_layout(chunk_rows, v) > ws_bytes) return A3PO_ERR_WORKSPACE;
+  __nv_bfloat16* dz = static_cast<__nv_bfloat16*>(ws);  // [chunk_rows, vpad]
   const int vpad = static_cast<int>(round_up(static_cast<size_t>(v), 8));
 
-  A3PO_RETURN_IF(transpose_bf16(w, v, h, h, wt, vpad, stream));  // W^T [h, vpad]
   for (long long r0 = 0; r0 < n; r0 += chunk_rows) {
     const long long r1 = (r0 + chunk_rows < n) ? r0 + chunk_rows : n;
     const long long nc = r1 - r0;
     const __nv_bfloat16* hid_c = hidden + r0 * h;
-    A3PO_RETURN_IF(transpose_bf16(hid_c, nc, h, h, ht, chunk_rows, stream));  // hidden^T [h, chunk]
-    // dz chunk (and its transpose) from recomputed logits
-    DzEpilogue::Params dp{targets, lse, grad_logp, r0, r1, v, vpad, chunk_rows, inv_t * kLog2e, inv_t, dz, dzt};
-    A3PO_RETURN_IF(launch_gemm<DzEpilogue>(hid_c, nc, h, w, v, h, h, 0, dp, status, stream));
-    // grad_hidden[r0:r1, :] = dz [nc, v] * (W^T [h, v])^T
+    // dz[t, v] for this chunk of rows, from recomputed logits:  A = hidden (K-major), B = W (K-major)
+    DzEpilogue::Params dp{targets, lse, grad_logp, r0, r1, v, vpad, inv_t * kLog2e, inv_t, dz};
+    A3PO_RETURN_IF((launch_gemm<DzEpilogue, false, false>(Operand{hid_c, nc, h, h}, Operand{w, v, h, h}, 0, dp,
+                                                          status, stream)));
+    // grad_hidden[t, j] = sum_v dz[t, v] W[v, j]:  A = dz (K = v contiguous), B = W read N-major
     StoreBf16Epilogue::Params hp{grad_hidden + r0 * h, h, nc, h};
-    A3PO_RETURN_IF(launch_gemm<StoreBf16Epilogue>(dz, nc, vpad, wt, h, vpad, v, 0, hp, status, stream));
-    // grad_w (+)= dz^T [v, nc] * (hidden^T [h, nc])^T
+    A3PO_RETURN_IF((launch_gemm<StoreBf16Epilogue, false, true>(Operand{dz, nc, v, vpad}, Operand{w, h, v, h}, 0, hp,
+                                                                status, stream)));
+    // grad_w[v, j] (+)= sum_t dz[t, v] hidden[t, j]:  A = dz read M-major, B = hidden read N-major (K = t)
     StoreF32Epilogue::Params wp{grad_w, h, v, h, (accumulate || r0 > 0) ? 1 : 0};
-    A3PO_RETURN_IF(launch_gemm<StoreF32Epilogue>(dzt, v, chunk_rows, ht, h, chunk_rows, nc, 0, wp, status, stream));
+    A3PO_RETURN_IF((launch_gemm<StoreF32Epilogue, true, true>(Operand{dz, v, nc, vpad}, Operand{hid_c, h, nc, h}, 0,
+                                                              wp, status, stream)));
   }
   return A3PO_OK;
 }

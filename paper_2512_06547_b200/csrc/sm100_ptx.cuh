@@ -152,11 +152,29 @@ __device__ __forceinline__ uint64_t umma_desc_k_major_sw128(uint32_t smem_addr) 
   return d;
 }
 
-// Instruction descriptor, kind::f16: bf16 x bf16 -> fp32, both operands K-major, tile M x N.
-__host__ __device__ constexpr uint32_t umma_idesc_bf16_f32(int m, int n) {
+// Shared-memory matrix descriptor for an MN-major bf16 tile (the M or N index is the contiguous
+// one) stored with the 128-byte swizzle: each 128-byte row holds 64 consecutive M/N elements of
+// one k; eight k rows form a 1024-byte swizzle atom; atoms of consecutive k groups follow every
+// 1024 bytes (stride byte offset) and the next block of 64 M/N elements starts `mn_block_bytes`
+// further (leading byte offset).  One UMMA (K = 16) spans two k groups.
+__device__ __forceinline__ uint64_t umma_desc_mn_major_sw128(uint32_t smem_addr, uint32_t mn_block_bytes) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((smem_addr & 0x3ffffu) >> 4);
+  d |= static_cast<uint64_t>((mn_block_bytes >> 4) & 0x3fffu) << 16;  // leading byte offset
+  d |= static_cast<uint64_t>(1024 >> 4) << 32;                         // stride byte offset
+  d |= static_cast<uint64_t>(1) << 46;
+  d |= static_cast<uint64_t>(2) << 61;
+  return d;
+}
+
+// Instruction descriptor, kind::f16: bf16 x bf16 -> fp32, tile M x N; a_mn / b_mn select an
+// MN-major (transposed) shared-memory operand instead of the K-major default.
+__host__ __device__ constexpr uint32_t umma_idesc_bf16_f32(int m, int n, bool a_mn = false, bool b_mn = false) {
   return (1u << 4)                              // D format: fp32
          | (1u << 7)                            // A format: bf16
          | (1u << 10)                           // B format: bf16
+         | (a_mn ? (1u << 15) : 0u)             // A major-ness
+         | (b_mn ? (1u << 16) : 0u)             // B major-ness
          | (static_cast<uint32_t>(n >> 3) << 17)  // N / 8
          | (static_cast<uint32_t>(m >> 4) << 24); // M / 16
 }
