@@ -40,7 +40,8 @@ typedef enum {
   A3PO_ERR_UNSUPPORTED = -2,  /* dtype/shape/alignment the kernels do not handle                */
   A3PO_ERR_WORKSPACE = -3,    /* ws is NULL, misaligned or smaller than the minimum             */
   A3PO_ERR_CUDA = -4,         /* a CUDA runtime/driver call or a kernel launch failed           */
-  A3PO_ERR_NO_DEVICE = -5     /* no usable sm_100 device is current                             */
+  A3PO_ERR_NO_DEVICE = -5,    /* no usable sm_100 device is current                             */
+  A3PO_ERR_TOO_LARGE = -6     /* N exceeds the fixed scratch of a3po_loss_fwd_static            */
 } a3po_error;
 
 /* Storage type of hidden, W and grad_hidden.  Accumulation is always fp32. */
@@ -172,6 +173,40 @@ int a3po_loss_fwd_bwd(const float* logp, const float* behav_logp, const int32_t*
                       int32_t current_version, const float* adv, const uint8_t* mask, int64_t N,
                       float clip_eps, int detach_prox, float* loss, a3po_stats* stats,
                       float* grad_logp, void* ws, size_t ws_bytes, void* stream);
+
+/* --------------------------------------------------------------------------------------------
+ * a3po_loss_fwd for callers that have no way to hand over a workspace (the paper has no
+ * counterpart: this is a packaging variant, the arithmetic is a3po_loss_fwd's).
+ *
+ * Who needs it: code that runs where device memory cannot be obtained at call time — a hook
+ * inside a host framework whose memory pool is the only permitted allocator and is not exposed
+ * to the hook, a latency-critical loop in which an allocation (an implicit device-wide
+ * synchronisation) is forbidden, or a process whose device memory has been carved up in advance
+ * and where cudaMalloc simply fails.  Such a caller still owns its inputs and outputs; what it
+ * lacks is the few megabytes of scratch the loss kernels reduce through.
+ *
+ * Here that scratch is a fixed array inside the library's device image (about 4.2 MiB, sized
+ * for A3PO_LOSS_FWD_STATIC_MAX_TOKENS tokens).  Every GPU on which the library is loaded holds
+ * it from load until the process exits, whether or not this function is ever called.  The
+ * function calls no cudaMalloc / cudaFree and no allocating library routine (with the optional
+ * per-kernel profile left off, which is the default, it creates no CUDA objects at all).
+ *
+ * Arguments, outputs and error codes are those of a3po_loss_fwd without ws / ws_bytes, plus:
+ *   - N > A3PO_LOSS_FWD_STATIC_MAX_TOKENS returns A3PO_ERR_TOO_LARGE before anything is
+ *     launched or written; use a3po_loss_fwd with a caller workspace for larger batches.
+ *   - The first call on each device looks up the array's device address (once per device, with
+ *     that device current).  That first call should be made before any stream capture begins.
+ *   - All calls on one device share the one array.  Nothing in it has to be zero on entry: a call
+ *     reads only words it has written itself, so the previous call's leftovers are harmless.
+ *     But two calls whose kernels overlap on the GPU (different streams, or different host
+ *     threads without ordering) race on it and corrupt each other's result: serialise them.
+ * ------------------------------------------------------------------------------------------ */
+#define A3PO_LOSS_FWD_STATIC_MAX_TOKENS (1 << 20)
+
+int a3po_loss_fwd_static(const float* logp, const float* behav_logp, const int32_t* versions,
+                         int versions_per_seq, const int32_t* cu_seqlens, int B,
+                         int32_t current_version, const float* adv, const uint8_t* mask, int64_t N,
+                         float clip_eps, float* loss, a3po_stats* stats, void* stream);
 
 /* --------------------------------------------------------------------------------------------
  * One whole training-step pass with per-step inputs in HOST memory (no counterpart in the

@@ -13,6 +13,7 @@ from .binding import (  # noqa: F401
     a3po_loss_bwd,
     a3po_loss_fwd,
     a3po_loss_fwd_bwd,
+    a3po_loss_fwd_static,
     a3po_loss_workspace_bytes,
     a3po_profile_enable,
     a3po_profile_read,

@@ -49,6 +49,8 @@ _SIGNATURES = {
                                         c_float, c_void_p, c_void_p, c_int, c_void_p, c_size_t, c_void_p, c_void_p]),
     "a3po_loss_fwd": (c_int, [c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_int, c_int32, c_void_p, c_void_p,
                               c_int64, c_float, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
+    "a3po_loss_fwd_static": (c_int, [c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_int, c_int32, c_void_p, c_void_p,
+                                     c_int64, c_float, c_void_p, c_void_p, c_void_p]),
     "a3po_loss_bwd": (c_int, [c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_int, c_int32, c_void_p, c_void_p,
                               c_int64, c_float, c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
     "a3po_loss_fwd_bwd": (c_int, [c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_int, c_int32, c_void_p, c_void_p,
@@ -235,6 +237,21 @@ def a3po_loss_fwd(logp, behav_logp, versions, current_version, adv, mask, clip_e
                                       int(current_version), _ptr(adv), _ptr(mask), n, float(clip_eps), _ptr(loss),
                                       _ptr(stats), _ptr(ws), ws.numel(), _stream(stream))
     _check("a3po_loss_fwd", rc)
+
+
+LOSS_FWD_STATIC_MAX_TOKENS = 1 << 20
+
+
+def a3po_loss_fwd_static(logp, behav_logp, versions, current_version, adv, mask, clip_eps, loss, *, stats=None,
+                         cu_seqlens=None, stream=None):
+    """a3po_loss_fwd for callers that cannot supply a workspace: the scratch is a fixed array inside the
+    library (at most LOSS_FWD_STATIC_MAX_TOKENS tokens; calls on one device must not overlap)."""
+    n, per_seq, b = _loss_common(logp, behav_logp, versions, adv, mask, cu_seqlens)
+    _want(loss, torch.float32, "loss"); _want(stats, torch.uint8, "stats")
+    rc = load_library().a3po_loss_fwd_static(_ptr(logp), _ptr(behav_logp), _ptr(versions), per_seq, _ptr(cu_seqlens),
+                                             b, int(current_version), _ptr(adv), _ptr(mask), n, float(clip_eps),
+                                             _ptr(loss), _ptr(stats), _stream(stream))
+    _check("a3po_loss_fwd_static", rc)
 
 
 def a3po_loss_bwd(logp, behav_logp, versions, current_version, adv, mask, clip_eps, grad_logp, ws, *,

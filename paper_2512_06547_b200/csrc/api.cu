@@ -178,6 +178,7 @@ const char* a3po_status_string(int code) {
     case A3PO_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
     case A3PO_ERR_CUDA: return "CUDA call or kernel launch failed";
     case A3PO_ERR_NO_DEVICE: return "no usable CUDA device is current";
+    case A3PO_ERR_TOO_LARGE: return "N exceeds the fixed scratch of a3po_loss_fwd_static (A3PO_LOSS_FWD_STATIC_MAX_TOKENS)";
     default: return "unknown a3po status";
   }
 }

@@ -8,6 +8,8 @@
 // -> per-block partial -> one finalising block, in a fixed order, so results do not change from
 // run to run.
 
+#include <mutex>
+
 #include "a3po_common.cuh"
 
 namespace a3po {
@@ -364,6 +366,66 @@ int a3po_loss_fwd(const float* logp, const float* behav_logp, const int32_t* ver
                   size_t ws_bytes, void* stream) {
   return a3po::run_loss(a3po::kFwd, logp, behav_logp, versions, versions_per_seq, cu_seqlens, B, current_version,
                         adv, mask, N, clip_eps, 1, nullptr, nullptr, loss, stats, nullptr, ws, ws_bytes, stream);
+}
+
+}  // extern "C"
+
+// ---------------------------------------------------------------------------------------------------
+// Loss forward without a caller workspace: the scratch lives in this library's device image.
+// ---------------------------------------------------------------------------------------------------
+namespace a3po {
+namespace {
+
+constexpr size_t static_round(size_t x) { return (x + 255) / 256 * 256; }
+// Same layout as loss_ws_bytes(A3PO_LOSS_FWD_STATIC_MAX_TOKENS): block partials, block counts, M,
+// expanded per-token versions (checked against loss_ws_bytes at run time).
+constexpr size_t kStaticScratchBytes =
+    static_round(sizeof(LossPartial) * kMaxLossBlocks) + static_round(sizeof(long long) * kMaxLossBlocks) + 256 +
+    static_round(sizeof(int32_t) * static_cast<size_t>(A3PO_LOSS_FWD_STATIC_MAX_TOKENS)) + 256;
+
+// One copy per GPU that loads the library, resident until the process exits.  In host code this
+// name is only a handle for cudaGetSymbolAddress; it is not a device address.
+static __device__ __align__(256) unsigned char g_static_loss_scratch[kStaticScratchBytes];
+
+// Device address of the array on the current device, looked up once per device.
+int static_loss_scratch(void** out) {
+  static std::mutex mu;
+  static void* cached[64];
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
+    cudaGetLastError();
+    return A3PO_ERR_NO_DEVICE;
+  }
+  std::lock_guard<std::mutex> lock(mu);
+  if (!cached[dev]) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_loss_scratch) != cudaSuccess || !p) {
+      cudaGetLastError();
+      return A3PO_ERR_CUDA;
+    }
+    cached[dev] = p;
+  }
+  *out = cached[dev];
+  return A3PO_OK;
+}
+
+}  // namespace
+}  // namespace a3po
+
+extern "C" {
+
+int a3po_loss_fwd_static(const float* logp, const float* behav_logp, const int32_t* versions, int versions_per_seq,
+                         const int32_t* cu_seqlens, int B, int32_t current_version, const float* adv,
+                         const uint8_t* mask, int64_t N, float clip_eps, float* loss, a3po_stats* stats,
+                         void* stream) {
+  if (N > A3PO_LOSS_FWD_STATIC_MAX_TOKENS) return A3PO_ERR_TOO_LARGE;
+  if (N >= 0 && a3po::loss_ws_bytes(N) > a3po::kStaticScratchBytes) return A3PO_ERR_TOO_LARGE;
+  if (a3po::sm_count() <= 0) return A3PO_ERR_NO_DEVICE;
+  void* scratch = nullptr;
+  A3PO_RETURN_IF(a3po::static_loss_scratch(&scratch));
+  return a3po::run_loss(a3po::kFwd, logp, behav_logp, versions, versions_per_seq, cu_seqlens, B, current_version,
+                        adv, mask, N, clip_eps, 1, nullptr, nullptr, loss, stats, nullptr, scratch,
+                        a3po::kStaticScratchBytes, stream);
 }
 
 int a3po_loss_bwd(const float* logp, const float* behav_logp, const int32_t* versions, int versions_per_seq,
