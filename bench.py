@@ -56,8 +56,16 @@ class ClockSampler:
     def __init__(self, gpu_index: int):
         self.gpu_index = gpu_index
         self.proc = None
-        self.lines = []
+        self.lines = []          # (arrival time, csv line)
         self.thread = None
+        self.t_begin = None
+        self.t_end = None
+
+    def mark_begin(self):
+        self.t_begin = time.monotonic()
+
+    def mark_end(self):
+        self.t_end = time.monotonic()
 
     def start(self):
         try:
@@ -73,7 +81,7 @@ class ClockSampler:
 
     def _pump(self):
         for line in self.proc.stdout:
-            self.lines.append(line.strip())
+            self.lines.append((time.monotonic(), line.strip()))
 
     def stop(self):
         if self.proc is None:
@@ -85,7 +93,9 @@ class ClockSampler:
             self.proc.kill()
         sm, mx, power, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for ln in self.lines:
+        window = [ln for t, ln in self.lines
+                  if (self.t_begin is None or t >= self.t_begin + 0.05) and (self.t_end is None or t <= self.t_end)]
+        for ln in (window or [ln for _, ln in self.lines]):
             f = [x.strip() for x in ln.split(",")]
             if len(f) < 9:
                 continue
@@ -98,9 +108,8 @@ class ClockSampler:
                     reasons.add(name)
         if not sm:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
-        busy = [c for c, p in zip(sm, power) if p > 0.5 * max(power)] or sm
-        return {"sm_mhz": statistics.median(busy), "sm_max_mhz": max(mx), "power_w_max": max(power),
-                "samples": len(sm), "reasons": sorted(reasons)}
+        return {"sm_mhz": statistics.median(sm), "sm_min_mhz": min(sm), "sm_max_mhz": max(mx),
+                "power_w_max": max(power), "samples": len(sm), "reasons": sorted(reasons)}
 
 
 WORKLOAD_TEXT = {
@@ -204,7 +213,8 @@ def run_ours(args):
 
     # every rank draws its own shard of sequences (same shapes): weak scaling, no data-path collective
     seed = workloads.BASE_SEED + workloads._SEED_OFFSET[args.workload] + 1000 * rank
-    wl = workloads.make_workload(args.workload, dev, seed=seed)
+    shrink = dict(n_prompts=1, group=4) if args.small else {}   # --small: 4 sequences, for profiler captures
+    wl = workloads.make_workload(args.workload, dev, seed=seed, **shrink)
     n, h, v = wl.N, wl.H, wl.V
     dt = a3po.A3PO_BF16 if wl.dtype == "bf16" else a3po.A3PO_F32
     to_dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(dev)
@@ -234,24 +244,26 @@ def run_ours(args):
         a3po.a3po_token_logprobs_bwd(wl.hidden, wl.w, targets, lse, grad_logp, grad_hidden, grad_w, ws,
                                      status=status)
 
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()          # started early: nvidia-smi needs a moment before its first sample
     for _ in range(args.warmup):
         step()
     barrier()
 
     # ---- timed region: device-resident inputs
-    sampler = ClockSampler(local_rank)
-    if rank == 0:
-        sampler.start()
     a3po.a3po_profile_enable(True)
     a3po.a3po_profile_read()
     launches0 = a3po.a3po_kernel_launch_count()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
+    sampler.mark_begin()
     e0.record()
     for _ in range(args.steps):
         step()
     e1.record()
     barrier()
+    sampler.mark_end()
     launches = a3po.a3po_kernel_launch_count() - launches0
     a3po.a3po_profile_enable(False)
     per_kernel = a3po.a3po_profile_read()
@@ -351,7 +363,8 @@ def run_ours(args):
         "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16" if wl.dtype == "bf16" else "f32", "data": "synthetic",
-        "config": {"workload": WORKLOAD_TEXT[args.workload], "rows_per_gpu": n, "valid_tokens_per_gpu": n_valid,
+        "config": {"workload": WORKLOAD_TEXT[args.workload] + (" [--small: 4 sequences only]" if args.small else ""),
+                   "rows_per_gpu": n, "valid_tokens_per_gpu": n_valid,
                    "H": h, "V": v, "parallelism": f"dp{world} (independent shards)",
                    "l2": "no flush: W (%.0f MB) and the dz scratch are larger than the 126 MB L2"
                          % (v * h * 2 / 1e6)},
@@ -371,17 +384,104 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+# ------------------------------------------------------------------------------------ loss-only sweep
+def run_loss_sweep(args):
+    """Loss kernels alone on the bandwidth-sweep workload: fwd, bwd and fused fwd+bwd at --tokens tokens.
+    Every iteration is timed with its own CUDA-event pair; when the inputs are smaller than 2x L2 a 512 MB
+    buffer is overwritten between iterations (untimed) to flush L2."""
+    import numpy as np
+    import torch
+
+    import paper_2512_06547_b200 as a3po
+    from paper_2512_06547_b200 import workloads
+
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    n = args.tokens
+    inp = workloads.loss_sweep(n)
+    to_dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(dev)
+    logp, behav, versions, adv, mask = (to_dev(inp[k]) for k in ("logp", "behav_logp", "versions", "adv", "mask"))
+    common = (logp, behav, versions, inp["current_version"], adv, mask, inp["clip_eps"])
+    ws = a3po.new_workspace(a3po.a3po_loss_workspace_bytes(n), dev)
+    loss = torch.zeros(1, device=dev)
+    stats = a3po.new_stats(dev)
+    grad = torch.empty(n, device=dev)
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev) if 21 * n < (256 << 20) else None
+    calls = {
+        "fwd": (lambda: a3po.a3po_loss_fwd(*common, loss, ws, stats=stats), 17),
+        "bwd": (lambda: a3po.a3po_loss_bwd(*common, grad, ws, fwd_stats=stats), 21),
+        "fwd_bwd": (lambda: a3po.a3po_loss_fwd_bwd(*common, loss, grad, ws, stats=stats), 22),
+    }
+    peaks = load_peaks()
+    sampler = ClockSampler(0)
+    sampler.start()
+    results = {}
+    a3po.a3po_profile_enable(True)
+    sampler_marked = False
+    for name, (fn, bytes_per_token) in calls.items():
+        for _ in range(max(args.warmup, 3)):
+            fn()
+        torch.cuda.synchronize()
+        a3po.a3po_profile_read()
+        if not sampler_marked:
+            sampler.mark_begin()
+            sampler_marked = True
+        call_ms = []
+        for _ in range(args.steps):
+            if flush is not None:
+                flush.fill_(1)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn()
+            e1.record()
+            torch.cuda.synchronize()
+            call_ms.append(e0.elapsed_time(e1))
+        prof = a3po.a3po_profile_read()
+        main_ms = [ms for k, ms in prof if k in ("loss_fwd", "loss_bwd", "loss_fwd_bwd")]
+        kernel_ms = statistics.mean(main_ms)
+        main_bytes = bytes_per_token - (1 if name == "fwd_bwd" else 0)     # the mask pre-count is its own kernel
+        results[name] = {
+            "call_ms": statistics.mean(call_ms), "kernel_ms": kernel_ms, "launches_per_call": len(prof) // args.steps,
+            "algorithmic_bytes_per_token": bytes_per_token,
+            "call_gbs": bytes_per_token * n / (statistics.mean(call_ms) * 1e-3) / 1e9,
+            "kernel_gbs": main_bytes * n / (kernel_ms * 1e-3) / 1e9,
+        }
+    sampler.mark_end()
+    a3po.a3po_profile_enable(False)
+    clocks = sampler.stop()
+    best = results["fwd_bwd"]
+    line = {
+        "metric": METRIC, "value": n / (best["call_ms"] * 1e-3), "unit": "tokens/s", "n_gpus": 1, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": best["call_ms"], "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"loss-only bandwidth sweep, N={n} tokens: fp32 logp / behaviour logp ~ -Exp(1), int32 "
+                               "per-token versions (staleness U{0..8}), fp32 advantage, uint8 mask (90% kept), eps=0.2",
+                   "l2": "flushed between iterations" if flush is not None else "inputs exceed L2"},
+        "roofline": {"bound": "hbm", "kernel": "loss_fwd_bwd", "achieved": round(best["kernel_gbs"], 1),
+                     "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": round(best["kernel_gbs"] / peaks["hbm_gbs"], 4),
+                     "frac_of_nominal_8000": round(best["kernel_gbs"] / 8000.0, 4), "traffic": None,
+                     "peak_source": f"{peaks['_source']} copy bandwidth"},
+        "loss_kernels": results, "clocks": clocks, "gpu_launches": None, "e2e": None, "cpu_baseline": None,
+    }
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="1p5b", choices=sorted(WORKLOAD_TEXT))
+    ap.add_argument("--workload", default="1p5b", choices=sorted(WORKLOAD_TEXT) + ["loss_sweep"])
+    ap.add_argument("--tokens", type=int, default=1 << 26, help="token count of --workload loss_sweep")
     ap.add_argument("--oracle-rows", type=int, default=256)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--small", action="store_true",
+                    help="same shapes with 4 sequences only (a profiler-sized case; not a benchmark number)")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.workload == "loss_sweep":
+        run_loss_sweep(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         if args.warmup < 3:
