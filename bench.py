@@ -189,6 +189,25 @@ def run_reference(args):
 
 
 # ------------------------------------------------------------------------------------ our arm
+def rank_seed(workload: str, rank: int) -> int:
+    """Every rank draws its own shard of sequences (same shapes, different draws): weak scaling."""
+    from paper_2512_06547_b200 import workloads
+    return workloads.BASE_SEED + workloads._SEED_OFFSET[workload] + 1000 * rank
+
+
+def reduce_over_ranks(times_ms, counts, device):
+    """Whole-job figures: MAX over ranks of each time, SUM over ranks of each count.
+    Works with any initialised process group (nccl on GPUs, gloo in the CPU test) or none."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(times_ms), dtype=torch.float64, device=device)
+    c = torch.tensor(list(counts), dtype=torch.float64, device=device)
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.all_reduce(c, op=dist.ReduceOp.SUM)
+    return t.tolist(), c.tolist()
+
+
 def run_ours(args):
     import numpy as np
     import torch
@@ -212,7 +231,7 @@ def run_ours(args):
         torch.cuda.synchronize()
 
     # every rank draws its own shard of sequences (same shapes): weak scaling, no data-path collective
-    seed = workloads.BASE_SEED + workloads._SEED_OFFSET[args.workload] + 1000 * rank
+    seed = rank_seed(args.workload, rank)
     shrink = dict(n_prompts=1, group=4) if args.small else {}   # --small: 4 sequences, for profiler captures
     wl = workloads.make_workload(args.workload, dev, seed=seed, **shrink)
     n, h, v = wl.N, wl.H, wl.V
@@ -302,13 +321,8 @@ def run_ours(args):
     d2h = 4 + 24
 
     # ---- max over ranks
-    times = torch.tensor([ms_total, e2e_ms_total], dtype=torch.float64, device=dev)
-    counts = torch.tensor([float(n_valid), float(n)], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-        dist.all_reduce(counts, op=dist.ReduceOp.SUM)
-    ms_total, e2e_ms_total = times.tolist()
-    total_valid, total_rows = counts.tolist()
+    (ms_total, e2e_ms_total), (total_valid, total_rows) = reduce_over_ranks(
+        [ms_total, e2e_ms_total], [float(n_valid), float(n)], dev)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()

@@ -18,6 +18,7 @@
 // Every mbarrier wait is bounded; on expiry the CTA raises A3PO_STATUS_WAIT_TIMEOUT in the
 // caller's status word, releases its TMEM and exits.
 
+#include <cstring>
 #include <mutex>
 
 #include "a3po_common.cuh"
@@ -40,7 +41,8 @@ constexpr uint32_t kBBytes = BN * BK * 2;
 constexpr uint32_t kStageBytes = kABytes + kBBytes;
 constexpr uint32_t kMnBlockBytes = 64 * BK * 2;  // one 64 (M/N) x 64 (k) box of an MN-major operand
 constexpr uint32_t kTmemCols = 512;
-constexpr size_t kSmemBytes = 1024 /*alignment slack*/ + kStages * kStageBytes + 256 /*barriers*/;
+constexpr uint32_t kSlabBytes = BM * 128;  // output staging slab: 128 rows x 128 bytes
+constexpr size_t kSmemBytes = 1024 /*alignment slack*/ + kStages * kStageBytes + 2 * kSlabBytes + 256 /*barriers*/;
 constexpr int kGroupM = 16;
 
 // Work decomposition: an item is (row tile, vocabulary split); a split is a contiguous range of
@@ -87,10 +89,49 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&p);
 }
 
+// ------------------------------------------------------------------------------------ tensor maps
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static std::once_flag once;
+  static EncodeTiledFn fn = nullptr;
+  std::call_once(once, [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+    else
+      cudaGetLastError();
+  });
+  return fn;
+}
+
+
+// Tensor map of an output matrix [rows, cols] (row-major, `pitch` elements per row, 2- or 4-byte
+// elements) for slab stores: boxes of 128 rows x 128 bytes with the 128-byte swizzle.
+int make_out_map(CUtensorMap* map, const void* base, int elt_bytes, long long cols, long long rows, long long pitch) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return A3PO_ERR_CUDA;
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(pitch) * elt_bytes};
+  const cuuint32_t box[2] = {static_cast<cuuint32_t>(128 / elt_bytes), static_cast<cuuint32_t>(BM)};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = fn(map, elt_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
+                        const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                        CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? A3PO_OK : A3PO_ERR_CUDA;
+}
+
 // ------------------------------------------------------------------------------------ epilogues
 // Each epilogue thread owns one accumulator row (`row` = global row of the A operand).
 // begin(): per-item state; chunk(): 32 consecutive fp32 columns starting at global column `col0`;
 // end(): per-item output.
+
+struct SlabStore;  // output staging for TMA stores, defined below
 
 template <bool ENT>
 struct FwdEpilogue {
@@ -105,14 +146,21 @@ struct FwdEpilogue {
     float* part_ent;
     float* zy;
   };
+  static int make_c_map(const Params&, CUtensorMap* map) {
+    memset(map, 0, sizeof(*map));  // the forward stores nothing through the copy engine
+    return A3PO_OK;
+  }
   float m, s, e;
   int y;
-  __device__ __forceinline__ void begin(const Params& p, long long row) {
+  long long row;
+  __device__ __forceinline__ void begin(const Params& p, long long row_) {
+    row = row_;
     m = -INFINITY; s = 0.f; e = 0.f;
     y = -1;
     if (row < p.n) y = min(max(p.targets[row], 0), p.v - 1);
   }
-  __device__ __forceinline__ void chunk(const Params& p, long long row, int col0, uint32_t (&r)[kEpiChunk]) {
+  __device__ __forceinline__ void chunk(const Params& p, int /*tile_row0*/, int col0, uint32_t (&r)[kEpiChunk],
+                                        SlabStore&) {
     if (col0 + kEpiChunk > p.v) {  // ragged vocabulary tail: columns past V do not exist
 #pragma unroll
       for (int j = 0; j < kEpiChunk; ++j)
@@ -154,6 +202,48 @@ struct FwdEpilogue {
   }
 };
 
+// Staging of output tiles for TMA stores.  The 128 epilogue threads fill a 128-row x 128-byte
+// slab in shared memory (one row each, 128-byte swizzle), and one of them hands the slab to the
+// copy engine, which writes it to global memory fully coalesced and clips it at the tensor's
+// extents (ragged row / column tails need no guards).  Two slabs alternate so that filling one
+// overlaps the copy of the other.
+struct SlabStore {
+  uint8_t* slab0;
+  uint8_t* slab1;
+  const CUtensorMap* map;
+  int row_in_tile;
+  bool issuer;
+  uint32_t issued = 0;
+  static constexpr int kBarrierId = 1;
+
+  // Returns the slab to fill next; all epilogue threads call it together.
+  __device__ __forceinline__ uint8_t* acquire() {
+    if (issuer) bulk_wait_group_read<1>();  // the copy that used this slab two submissions ago has read it
+    named_barrier_sync(kBarrierId, 128);
+    return (issued & 1u) ? slab1 : slab0;
+  }
+  // 16-byte piece j (0..7) of this thread's row.
+  __device__ __forceinline__ uint4* piece(uint8_t* s, int j) const {
+    return reinterpret_cast<uint4*>(s + row_in_tile * 128 + ((j ^ (row_in_tile & 7)) << 4));
+  }
+  // Hands the filled slab to the copy engine: global tile origin (x, y) in elements.
+  __device__ __forceinline__ void submit(uint8_t* s, int x, int y, bool in_range, bool reduce_add) {
+    fence_proxy_async_smem();
+    named_barrier_sync(kBarrierId, 128);
+    if (issuer) {
+      if (in_range) {
+        if (reduce_add) tma_reduce_add_f32_2d(map, s, x, y);
+        else tma_store_2d(map, s, x, y);
+      }
+      bulk_commit_group();
+    }
+    ++issued;
+  }
+  __device__ __forceinline__ void drain() {
+    if (issuer) bulk_wait_group<0>();
+  }
+};
+
 struct DzEpilogue {
   static constexpr int kKernelId = kKTcDz;
   struct Params {
@@ -168,20 +258,23 @@ struct DzEpilogue {
     float inv_t;
     __nv_bfloat16* dz;        // [chunk rows, vpad]
   };
+  static int make_c_map(const Params& p, CUtensorMap* map) {
+    return make_out_map(map, p.dz, /*bytes per element*/ 2, p.v, p.row_end - p.row_begin, p.vpad);
+  }
   float g, l2;
   int y;
-  bool valid;
+  uint8_t* cur;
   __device__ __forceinline__ void begin(const Params& p, long long row) {
     const long long t = p.row_begin + row;
-    valid = t < p.row_end;
     g = 0.f; l2 = INFINITY; y = -1;
-    if (valid) {
+    if (t < p.row_end) {
       g = p.grad_logp[t] * p.inv_t;
       if (g != 0.f) l2 = p.lse[t] * kLog2e;   // g == 0: exp2(-inf) = 0, the row contributes nothing
       y = min(max(p.targets[t], 0), p.v - 1);
     }
   }
-  __device__ __forceinline__ void chunk(const Params& p, long long row, int col0, uint32_t (&r)[kEpiChunk]) {
+  __device__ __forceinline__ void chunk(const Params& p, int tile_row0, int col0, uint32_t (&r)[kEpiChunk],
+                                        SlabStore& st) {
     float d[kEpiChunk];
     const float ng = -g;
 #pragma unroll
@@ -192,20 +285,19 @@ struct DzEpilogue {
       for (int j = 0; j < kEpiChunk; ++j)
         if (col0 + j == y) d[j] += g;
     }
-    if (!valid) return;
-    // row-major copy: 64 contiguous bytes per thread
-    __nv_bfloat16* dst = p.dz + row * p.vpad + col0;
+    // a slab holds 64 bf16 columns: two consecutive 32-column chunks
+    const int half = (col0 >> 5) & 1;
+    if (half == 0) cur = st.acquire();
 #pragma unroll
-    for (int q = 0; q < kEpiChunk / 8; ++q) {
-      if (col0 + q * 8 < p.vpad) {
-        uint4 u;
-        u.x = pack_bf16x2(d[q * 8 + 0], d[q * 8 + 1]);
-        u.y = pack_bf16x2(d[q * 8 + 2], d[q * 8 + 3]);
-        u.z = pack_bf16x2(d[q * 8 + 4], d[q * 8 + 5]);
-        u.w = pack_bf16x2(d[q * 8 + 6], d[q * 8 + 7]);
-        *reinterpret_cast<uint4*>(dst + q * 8) = u;
-      }
+    for (int q = 0; q < 4; ++q) {
+      uint4 u;
+      u.x = pack_bf16x2(d[q * 8 + 0], d[q * 8 + 1]);
+      u.y = pack_bf16x2(d[q * 8 + 2], d[q * 8 + 3]);
+      u.z = pack_bf16x2(d[q * 8 + 4], d[q * 8 + 5]);
+      u.w = pack_bf16x2(d[q * 8 + 6], d[q * 8 + 7]);
+      *st.piece(cur, half * 4 + q) = u;
     }
+    if (half == 1) st.submit(cur, col0 - 32, tile_row0, col0 - 32 < p.v, false);
   }
   __device__ __forceinline__ void end(const Params&, long long, int) {}
 };
@@ -218,21 +310,25 @@ struct StoreBf16Epilogue {
     long long m_rows;
     int n_cols;  // multiple of 8
   };
+  static int make_c_map(const Params& p, CUtensorMap* map) {
+    return make_out_map(map, p.c, 2, p.n_cols, p.m_rows, p.ldc);
+  }
+  uint8_t* cur;
   __device__ __forceinline__ void begin(const Params&, long long) {}
-  __device__ __forceinline__ void chunk(const Params& p, long long row, int col0, uint32_t (&r)[kEpiChunk]) {
-    if (row >= p.m_rows) return;
-    __nv_bfloat16* dst = p.c + row * p.ldc + col0;
+  __device__ __forceinline__ void chunk(const Params& p, int tile_row0, int col0, uint32_t (&r)[kEpiChunk],
+                                        SlabStore& st) {
+    const int half = (col0 >> 5) & 1;
+    if (half == 0) cur = st.acquire();
 #pragma unroll
-    for (int q = 0; q < kEpiChunk / 8; ++q) {
-      if (col0 + q * 8 < p.n_cols) {
-        uint4 u;
-        u.x = pack_bf16x2(bits_to_float(r[q * 8 + 0]), bits_to_float(r[q * 8 + 1]));
-        u.y = pack_bf16x2(bits_to_float(r[q * 8 + 2]), bits_to_float(r[q * 8 + 3]));
-        u.z = pack_bf16x2(bits_to_float(r[q * 8 + 4]), bits_to_float(r[q * 8 + 5]));
-        u.w = pack_bf16x2(bits_to_float(r[q * 8 + 6]), bits_to_float(r[q * 8 + 7]));
-        *reinterpret_cast<uint4*>(dst + q * 8) = u;
-      }
+    for (int q = 0; q < 4; ++q) {
+      uint4 u;
+      u.x = pack_bf16x2(bits_to_float(r[q * 8 + 0]), bits_to_float(r[q * 8 + 1]));
+      u.y = pack_bf16x2(bits_to_float(r[q * 8 + 2]), bits_to_float(r[q * 8 + 3]));
+      u.z = pack_bf16x2(bits_to_float(r[q * 8 + 4]), bits_to_float(r[q * 8 + 5]));
+      u.w = pack_bf16x2(bits_to_float(r[q * 8 + 6]), bits_to_float(r[q * 8 + 7]));
+      *st.piece(cur, half * 4 + q) = u;
     }
+    if (half == 1) st.submit(cur, col0 - 32, tile_row0, col0 - 32 < p.n_cols, false);
   }
   __device__ __forceinline__ void end(const Params&, long long, int) {}
 };
@@ -244,27 +340,37 @@ struct StoreF32Epilogue {
     long long ldc;
     long long m_rows;
     int n_cols;  // multiple of 4
-    int accumulate;
+    int accumulate;  // add into c (performed by the copy engine's element-wise reduction) instead of overwriting
   };
+  static int make_c_map(const Params& p, CUtensorMap* map) {
+    return make_out_map(map, p.c, 4, p.n_cols, p.m_rows, p.ldc);
+  }
   __device__ __forceinline__ void begin(const Params&, long long) {}
-  __device__ __forceinline__ void chunk(const Params& p, long long row, int col0, uint32_t (&r)[kEpiChunk]) {
-    if (row >= p.m_rows) return;
-    float* dst = p.c + row * p.ldc + col0;
+  __device__ __forceinline__ void chunk(const Params& p, int tile_row0, int col0, uint32_t (&r)[kEpiChunk],
+                                        SlabStore& st) {
+    uint8_t* s = st.acquire();  // 32 fp32 columns = one 128-byte slab row
 #pragma unroll
-    for (int q = 0; q < kEpiChunk / 4; ++q) {
-      if (col0 + q * 4 < p.n_cols) {
-        float4 o = make_float4(bits_to_float(r[q * 4 + 0]), bits_to_float(r[q * 4 + 1]),
-                               bits_to_float(r[q * 4 + 2]), bits_to_float(r[q * 4 + 3]));
-        if (p.accumulate) {
-          const float4 old = *reinterpret_cast<const float4*>(dst + q * 4);
-          o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
-        }
-        *reinterpret_cast<float4*>(dst + q * 4) = o;
-      }
-    }
+    for (int q = 0; q < 8; ++q) *st.piece(s, q) = make_uint4(r[q * 4 + 0], r[q * 4 + 1], r[q * 4 + 2], r[q * 4 + 3]);
+    st.submit(s, col0, tile_row0, col0 < p.n_cols, p.accumulate != 0);
   }
   __device__ __forceinline__ void end(const Params&, long long, int) {}
 };
+
+// AND of a predicate over the 128 epilogue threads (hardware barrier 2).
+__device__ __forceinline__ bool all_epilogue_threads(bool pred) {
+  uint32_t out;
+  asm volatile(
+      "{\n"
+      ".reg .pred p, q;\n"
+      "setp.ne.u32 q, %1, 0;\n"
+      "bar.red.and.pred p, 2, 128, q;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(out)
+      : "r"(static_cast<uint32_t>(pred))
+      : "memory");
+  return out != 0;
+}
 
 // ------------------------------------------------------------------------------------ the kernel
 // A_MN / B_MN: the operand is read from a tensor whose contiguous index is M (resp. N) instead of
@@ -272,13 +378,15 @@ struct StoreF32Epilogue {
 // shared-memory matrix, so no transposed copy of the operand ever has to exist in memory.
 template <class Epi, bool A_MN, bool B_MN>
 __global__ void __launch_bounds__(kTcThreads, 1)
-gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, ItemMap im,
-               int k_blocks, typename Epi::Params ep, uint32_t* status) {
+gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+               const __grid_constant__ CUtensorMap map_c, ItemMap im, int k_blocks, typename Epi::Params ep,
+               uint32_t* status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* smem_a = smem;
   uint8_t* smem_b = smem + kStages * kABytes;
-  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + kStages * kStageBytes);
+  uint8_t* smem_slabs = smem + kStages * kStageBytes;  // two 16 KB output staging slabs
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem_slabs + 2 * kSlabBytes);
   uint64_t* empty_bar = full_bar + kStages;
   uint64_t* tmem_full_bar = empty_bar + kStages;
   uint64_t* tmem_empty_bar = tmem_full_bar + 2;
@@ -389,12 +497,20 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     int acc = 0;
     uint32_t acc_phase = 0;
     Epi epi;
+    SlabStore st;
+    st.slab0 = smem_slabs;
+    st.slab1 = smem_slabs + kSlabBytes;
+    st.map = &map_c;
+    st.row_in_tile = row_in_tile;
+    st.issuer = (threadIdx.x == 2 * kWarp);
     for (long long i = blockIdx.x; i < im.items && ok; i += gridDim.x) {
       const Item it = decode_item(im, i);
-      const long long row = static_cast<long long>(it.m_tile) * BM + row_in_tile;
-      epi.begin(ep, row);
+      const int tile_row0 = it.m_tile * BM;
+      epi.begin(ep, static_cast<long long>(tile_row0) + row_in_tile);
       for (int nt = it.n_begin; nt < it.n_end && ok; ++nt) {
-        if (!mbar_wait(&tmem_full_bar[acc], acc_phase, abort_flag)) { ok = false; break; }
+        // the four epilogue warps share named barriers further down: they must agree on giving up
+        ok = all_epilogue_threads(mbar_wait(&tmem_full_bar[acc], acc_phase, abort_flag));
+        if (!ok) break;
         tcgen05_fence_after_sync();
         const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(acc * BN);
 #pragma unroll 1
@@ -402,15 +518,16 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           uint32_t r[kEpiChunk];
           tmem_ld_32x32(taddr + static_cast<uint32_t>(c * kEpiChunk), r);
           tmem_ld_wait();
-          epi.chunk(ep, row, nt * BN + c * kEpiChunk, r);
+          epi.chunk(ep, tile_row0, nt * BN + c * kEpiChunk, r, st);
         }
         tcgen05_fence_before_sync();
         __syncwarp();
         if (lane == 0) mbar_arrive(&tmem_empty_bar[acc]);
         if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
       }
-      if (ok) epi.end(ep, row, it.split);
+      if (ok) epi.end(ep, static_cast<long long>(tile_row0) + row_in_tile, it.split);
     }
+    st.drain();  // shared memory must stay valid until the copy engine has read every submitted slab
   }
 
   if (!ok) {
@@ -427,25 +544,6 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 }
 
 // ------------------------------------------------------------------------------------ host side
-using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-  static std::once_flag once;
-  static EncodeTiledFn fn = nullptr;
-  std::call_once(once, [] {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-        q == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(p);
-    else
-      cudaGetLastError();
-  });
-  return fn;
-}
-
 // One GEMM operand as it lies in memory (bf16, row-major with `pitch` elements per row).
 //   K-major : tensor [mn_extent rows, k_extent cols]   -> boxes of tile_mn rows x 64 k
 //   MN-major: tensor [k_extent rows, mn_extent cols]   -> boxes of 64 k rows x 64 M/N elements
@@ -475,9 +573,10 @@ int make_map(CUtensorMap* map, const Operand& op, bool mn_major, int tile_mn) {
 template <class Epi, bool A_MN, bool B_MN>
 int launch_gemm(const Operand& a, const Operand& b, int splits, const typename Epi::Params& ep, uint32_t* status,
                 cudaStream_t stream) {
-  CUtensorMap map_a, map_b;
+  CUtensorMap map_a, map_b, map_c;
   A3PO_RETURN_IF(make_map(&map_a, a, A_MN, BM));
   A3PO_RETURN_IF(make_map(&map_b, b, B_MN, BN));
+  A3PO_RETURN_IF(Epi::make_c_map(ep, &map_c));
   ItemMap im;
   im.m_tiles = static_cast<int>((a.mn_extent + BM - 1) / BM);
   im.n_tiles = static_cast<int>((b.mn_extent + BN - 1) / BN);
@@ -494,7 +593,7 @@ int launch_gemm(const Operand& a, const Operand& b, int splits, const typename E
   if (grid > im.items) grid = im.items;
   if (grid < 1) return A3PO_OK;
   A3PO_LAUNCH(Epi::kKernelId, stream, (kernel<<<static_cast<unsigned>(grid), kTcThreads, kSmemBytes, stream>>>(
-                                          map_a, map_b, im, k_blocks, ep, status)));
+                                          map_a, map_b, map_c, im, k_blocks, ep, status)));
   return after_launch();
 }
 

@@ -16,7 +16,7 @@ namespace a3po {
 namespace {
 
 constexpr int kLossThreads = 256;
-constexpr int kBlocksPerSm = 8;
+constexpr int kBlocksPerSm = 4;   // resident blocks per SM at <= 64 registers per thread
 constexpr int kMaxLossBlocks = 4096;
 
 struct alignas(16) LossPartial {
@@ -56,32 +56,32 @@ struct Acc {
 // One token of Eq. 2-4.  iw and r are evaluated through the closed form of the theorem
 // (r = w^alpha, iw = w^(1-alpha), w = exp(l_theta - l_behav)): the same function as the literal
 // interpolation of Eq. 3 but conditioned on the small difference of the two log-probs.
+// Staleness is exact for any pair of int32 versions: a signed compare decides d >= 1 and the
+// unsigned difference is d itself in that case; d = 1 takes alpha = 1 without a reciprocal.
 template <int MODE>
 __device__ __forceinline__ void token(float lt, float lb, int ver, float a, bool valid,
                                       const LossArgs& p, float coef, float& fsum, Acc& acc,
                                       float& grad) {
-  long long d = static_cast<long long>(p.current_version) - static_cast<long long>(ver);
-  float alpha = (d >= 1) ? __frcp_rn(static_cast<float>(d)) : 1.0f;
-  float delta = lt - lb;
-  float ad = alpha * delta;
-  float r = fast_exp2(ad * kLog2e);
-  float iw = fast_exp2((delta - ad) * kLog2e);
-  float s1 = r * a;
-  float s2 = fminf(fmaxf(r, p.lo), p.hi) * a;
-  bool act = s1 <= s2;
-  float obj = iw * fminf(s1, s2);
+  const unsigned du = static_cast<unsigned>(p.current_version) - static_cast<unsigned>(ver);
+  const bool interpolate = (ver < p.current_version) && (du > 1u);
+  const float alpha = interpolate ? fast_rcp(static_cast<float>(du)) : 1.0f;
+  const float d2 = (lt - lb) * kLog2e;
+  const float ad2 = alpha * d2;
+  const float r = fast_exp2(ad2);
+  const float iw = fast_exp2(d2 - ad2);
+  const float s1 = r * a;
+  const float s2 = fminf(fmaxf(r, p.lo), p.hi) * a;
+  const bool act = s1 <= s2;
+  const float obj = iw * fminf(s1, s2);
   if (MODE != kBwd) {
-    if (valid) {
-      fsum += obj;
-      acc.n_valid += 1;
-      acc.n_clipped += act ? 0 : 1;
-      acc.iw_max = fmaxf(acc.iw_max, iw);
-      acc.iw_min = fminf(acc.iw_min, iw);
-    }
+    fsum += valid ? obj : 0.f;
+    acc.n_clipped += (valid && !act) ? 1 : 0;
+    acc.iw_max = fmaxf(acc.iw_max, valid ? iw : 0.f);
+    acc.iw_min = fminf(acc.iw_min, valid ? iw : 3.4e38f);
   }
   if (MODE != kFwd) {
-    float through = act ? iw * s1 : 0.f;
-    float dobj = p.detach ? through : fmaf(alpha, through - obj, obj);  // (1-a)*obj + a*through
+    const float through = act ? iw * s1 : 0.f;
+    const float dobj = p.detach ? through : fmaf(alpha, through - obj, obj);  // (1-a)*obj + a*through
     grad = valid ? coef * dobj : 0.f;
   }
 }
@@ -92,28 +92,35 @@ __device__ __forceinline__ void group4(long long g, const LossArgs& p, float coe
   const float4 lb = __ldcs(reinterpret_cast<const float4*>(p.behav) + g);
   const int4 ver = __ldcs(reinterpret_cast<const int4*>(p.versions) + g);
   const float4 a = __ldcs(reinterpret_cast<const float4*>(p.adv) + g);
-  const unsigned m = __ldcs(reinterpret_cast<const unsigned*>(p.mask) + g);
+  const unsigned m = __vcmpne4(__ldcs(reinterpret_cast<const unsigned*>(p.mask) + g), 0u);  // 0xff per valid token
   float fsum = 0.f;
   float4 gr;
   token<MODE>(lt.x, lb.x, ver.x, a.x, (m & 0x000000ffu) != 0, p, coef, fsum, acc, gr.x);
   token<MODE>(lt.y, lb.y, ver.y, a.y, (m & 0x0000ff00u) != 0, p, coef, fsum, acc, gr.y);
   token<MODE>(lt.z, lb.z, ver.z, a.z, (m & 0x00ff0000u) != 0, p, coef, fsum, acc, gr.z);
   token<MODE>(lt.w, lb.w, ver.w, a.w, (m & 0xff000000u) != 0, p, coef, fsum, acc, gr.w);
-  if (MODE != kBwd) acc.sum += static_cast<double>(fsum);
+  if (MODE != kBwd) {
+    acc.sum += static_cast<double>(fsum);
+    acc.n_valid += __popc(m) >> 3;
+  }
   if (MODE != kFwd) __stcs(reinterpret_cast<float4*>(p.grad_logp) + g, gr);
 }
 
 template <int MODE>
 __device__ __forceinline__ void single(long long t, const LossArgs& p, float coef, Acc& acc) {
   float fsum = 0.f, gr = 0.f;
-  token<MODE>(p.logp[t], p.behav[t], p.versions[t], p.adv[t], p.mask[t] != 0, p, coef, fsum, acc, gr);
-  if (MODE != kBwd) acc.sum += static_cast<double>(fsum);
+  const bool valid = p.mask[t] != 0;
+  token<MODE>(p.logp[t], p.behav[t], p.versions[t], p.adv[t], valid, p, coef, fsum, acc, gr);
+  if (MODE != kBwd) {
+    acc.sum += static_cast<double>(fsum);
+    acc.n_valid += valid ? 1 : 0;
+  }
   if (MODE != kFwd) p.grad_logp[t] = gr;
 }
 
 // VEC = true needs 16-byte aligned fp32/int32 arrays and a 4-byte aligned mask.
 template <int MODE, bool VEC>
-__global__ void __launch_bounds__(kLossThreads) loss_kernel(LossArgs p, LossPartial* partials) {
+__global__ void __launch_bounds__(kLossThreads, kBlocksPerSm) loss_kernel(LossArgs p, LossPartial* partials) {
   float coef = 0.f;
   if (MODE != kFwd) {
     long long m = *p.n_valid_ptr;

@@ -1,0 +1,108 @@
+"""GPU parity at the full sizes of the named configs, in the launch configuration bench.py times.
+
+A full fp64 oracle pass is out of reach there (the 8B-shaped forward alone is 1.6e14 flop), so:
+  * rows are independent: log-probs and grad_hidden are compared on sampled rows the oracle computes one by one;
+  * grad_w is compared exactly on a run whose upstream gradient is non-zero only on sampled rows spread over all
+    row tiles (the launch still sweeps the whole batch), and checked by a size-independent property (its sum
+    over the vocabulary vanishes) on the dense run;
+  * the loss stage is cheap for the oracle and is compared on every token.
+"""
+import numpy as np
+import pytest
+import torch
+
+import paper_2512_06547_b200 as a3po
+from oracle import a3po_oracle as orc
+from paper_2512_06547_b200 import workloads
+from tests.helpers import GRAD_FRO_RTOL, LOGP_TOL_BF16, check_loss_outputs, rel_fro, to_np64
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def _to_dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).to(DEV)
+
+
+def _run_fullsize(name, n_sample_rows, seed):
+    wl = workloads.make_workload(name, DEV)
+    n, h, v = wl.N, wl.H, wl.V
+    rng = np.random.default_rng(seed)
+    targets, mask = _to_dev(wl.targets), _to_dev(wl.mask)
+    ws = a3po.new_workspace(a3po.a3po_train_step_workspace_bytes(n, h, v, a3po.A3PO_BF16))
+    logp, lse = torch.empty(n, device=DEV), torch.empty(n, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+
+    # ---- forward, whole batch; sampled valid rows against the oracle
+    a3po.a3po_token_logprobs_fwd(wl.hidden, wl.w, targets, logp, lse, ws, row_mask=mask, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    valid_rows = np.flatnonzero(wl.mask)
+    # spread over the batch, and always include the first and last valid row (first / last row tile)
+    idx = np.unique(np.concatenate([valid_rows[[0, -1]], rng.choice(valid_rows, n_sample_rows - 2, replace=False)]))
+    idx_t = torch.from_numpy(idx).to(DEV)
+    hn, wn = to_np64(wl.hidden[idx_t]), to_np64(wl.w)
+    logp_ref, lse_ref = orc.token_logprobs_fwd(hn, wn, wl.targets[idx])
+    logp_h, lse_h = logp.cpu().numpy(), lse.cpu().numpy()
+    assert np.max(np.abs(logp_h[idx] - logp_ref)) <= LOGP_TOL_BF16
+    assert np.max(np.abs(lse_h[idx] - lse_ref)) <= LOGP_TOL_BF16
+    assert np.all(logp_h <= 0) and np.all(np.isfinite(logp_h))
+    assert not logp_h[wl.mask == 0].any() and not lse_h[wl.mask == 0].any()
+
+    # ---- loss stage on every token, fed with a seeded log-prob array (not the GPU's)
+    lp_in = np.minimum(-(np.log(v) + 0.5) + rng.standard_normal(n), 0).astype(np.float32)
+    inp = dict(logp=lp_in, behav_logp=workloads.behav_logp_from(lp_in, wl.behav_noise), versions=wl.versions,
+               current_version=wl.current_version, adv=wl.adv, mask=wl.mask, clip_eps=wl.clip_eps, N=n)
+    loss = torch.zeros(1, device=DEV)
+    stats = a3po.new_stats()
+    grad_logp = torch.empty(n, device=DEV)
+    a3po.a3po_loss_fwd_bwd(_to_dev(inp["logp"]), _to_dev(inp["behav_logp"]), _to_dev(wl.versions), wl.current_version,
+                           _to_dev(wl.adv), mask, wl.clip_eps, loss, grad_logp, ws, stats=stats)
+    torch.cuda.synchronize()
+    check_loss_outputs(inp, float(loss.item()), a3po.read_stats(stats), grad_logp.cpu().numpy())
+
+    # ---- backward, dense upstream gradient (the oracle's): sampled rows of grad_hidden, property of grad_w
+    g_dense = orc.loss_bwd(inp["logp"], inp["behav_logp"], wl.versions, wl.current_version, wl.adv, wl.mask,
+                           wl.clip_eps).astype(np.float32)
+    grad_hidden = torch.empty_like(wl.hidden)
+    grad_w = torch.empty((v, h), dtype=torch.float32, device=DEV)
+    a3po.a3po_token_logprobs_bwd(wl.hidden, wl.w, targets, lse, _to_dev(g_dense), grad_hidden, grad_w, ws,
+                                 status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    gh_ref, _ = orc.token_logprobs_bwd(hn, wn, wl.targets[idx], g_dense[idx].astype(np.float64))
+    assert rel_fro(to_np64(grad_hidden[idx_t]), gh_ref) <= GRAD_FRO_RTOL
+    zero_rows = torch.from_numpy(np.flatnonzero(g_dense == 0)[:4096]).to(DEV)
+    assert not grad_hidden[zero_rows].float().abs().sum().item()
+    col_sum = grad_w.sum(dim=0, dtype=torch.float64)
+    col_abs = grad_w.abs().sum(dim=0, dtype=torch.float64)
+    assert float((col_sum.abs() / col_abs.clamp_min(1e-30)).max()) <= 2e-2      # each dz row sums to zero
+    assert torch.isfinite(grad_w).all()
+
+    # ---- backward, upstream gradient only on the sampled rows: grad_w and grad_hidden exactly
+    g_sparse = np.zeros(n, dtype=np.float32)
+    g_sparse[idx] = rng.standard_normal(len(idx)).astype(np.float32) / len(idx)
+    a3po.a3po_token_logprobs_bwd(wl.hidden, wl.w, targets, lse, _to_dev(g_sparse), grad_hidden, grad_w, ws,
+                                 status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    gh_ref, gw_ref = orc.token_logprobs_bwd(hn, wn, wl.targets[idx], g_sparse[idx].astype(np.float64))
+    assert rel_fro(to_np64(grad_hidden[idx_t]), gh_ref) <= GRAD_FRO_RTOL
+    assert rel_fro(to_np64(grad_w), gw_ref) <= GRAD_FRO_RTOL
+    assert float(grad_hidden.float().abs().sum().item()) == pytest.approx(
+        float(grad_hidden[idx_t].float().abs().sum().item()), rel=1e-6)      # nothing outside the sampled rows
+
+
+def test_1p5b_full_size():
+    """H=1536, V=151936, 16 x 1024 rows: the benchmark's own workload and launch configuration."""
+    _run_fullsize("1p5b", 96, seed=1)
+
+
+def test_8b_full_size():
+    """H=4096, V=151936, 64 x 2048 rows (several 16384-row chunks in the backward)."""
+    _run_fullsize("8b", 48, seed=2)
+
+
+def test_8b_packed_full_size():
+    """Packed varlen batch, ~1.1 M tokens, H=4096, per-token mask drops, ragged last row tile."""
+    _run_fullsize("8b_packed", 48, seed=3)
