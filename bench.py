@@ -340,12 +340,20 @@ def run_ours(args):
         a[0] += 1
         a[1] += ms
     kernel_total = sum(x[1] for x in agg.values()) or 1.0
-    flops_per_launch = 2.0 * n * v * h            # every gemm_tn instantiation contracts N x V x H once per step
+    # Algorithmic flops per launch = 2 * (rows that take part) * V * H: the forward processes the rows with
+    # mask != 0, the three backward contractions the rows whose upstream gradient is non-zero (padding and
+    # clipped tokens are skipped by the library, so they are not counted as work).
+    fwd_rows = n_valid
+    bwd_rows = int((grad_logp != 0).sum().item())
+    rows_of = {"gemm_tn<fwd_logsoftmax>": fwd_rows, "gemm_tn<dz>": bwd_rows, "gemm_tn<grad_hidden>": bwd_rows,
+               "gemm_tn<grad_w>": bwd_rows}
+    step_flops = 2.0 * v * h * (fwd_rows + 3 * bwd_rows)
     kernels = []
     for name, (cnt, ms) in sorted(agg.items(), key=lambda kv: -kv[1][1]):
         entry = {"kernel": name, "launches": cnt, "ms_total": round(ms, 4), "share": round(ms / kernel_total, 4)}
         if name.startswith("gemm_tn"):
-            entry["tflops"] = round(flops_per_launch * cnt / (ms * 1e-3) / 1e12, 1)
+            entry["rows"] = rows_of.get(name, n)
+            entry["tflops"] = round(2.0 * entry["rows"] * v * h * cnt / (ms * 1e-3) / 1e12, 1)
         kernels.append(entry)
     dom = kernels[0]
     sustained = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
@@ -357,7 +365,7 @@ def run_ours(args):
                     "peak_burst": peaks["bf16_tflops"], "frac_of_burst": round(achieved / peaks["bf16_tflops"], 4),
                     "frac_of_nominal_2250": round(achieved / 2250.0, 4),
                     "all_gemm_tn_tflops": round(
-                        sum(flops_per_launch * k["launches"] for k in kernels if k["kernel"].startswith("gemm_tn")) /
+                        sum(2.0 * k["rows"] * v * h * k["launches"] for k in kernels if k["kernel"].startswith("gemm_tn")) /
                         (sum(k["ms_total"] for k in kernels if k["kernel"].startswith("gemm_tn")) * 1e-3) / 1e12, 1)}
     else:
         roofline = {"bound": "hbm", "kernel": dom["kernel"], "achieved": None, "peak": peaks["hbm_gbs"],
@@ -383,7 +391,8 @@ def run_ours(args):
                    "l2": "no flush: W (%.0f MB) and the dz scratch are larger than the 126 MB L2"
                          % (v * h * 2 / 1e6)},
         "rows_per_s": total_rows * args.steps / (ms_total * 1e-3),
-        "executed_tflops": round(8.0 * n * v * h * world / (ms_per_step * 1e-3) / 1e12, 1),
+        "executed_tflops": round(step_flops * world / (ms_per_step * 1e-3) / 1e12, 1),
+        "rows_processed": {"fwd": fwd_rows, "bwd": bwd_rows, "of": n},
         "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": e2e_ms_total / args.steps},
         "gpu_launches": int(launches),

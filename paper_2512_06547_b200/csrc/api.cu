@@ -87,30 +87,33 @@ constexpr long long kTcChunkRows = 16384;
 __global__ void __launch_bounds__(kMergeThreads)
 merge_partials_kernel(const SoftmaxPartial* __restrict__ part, const float* __restrict__ part_ent,
                       const float* __restrict__ zy, const int32_t* __restrict__ targets,
-                      const uint8_t* __restrict__ row_mask, long long n, int v, int splits, float* __restrict__ logp,
-                      float* __restrict__ lse, float* __restrict__ entropy, uint32_t* status) {
+                      const uint8_t* __restrict__ row_mask, const int* __restrict__ pos, long long n, int v,
+                      int splits, float* __restrict__ logp, float* __restrict__ lse, float* __restrict__ entropy,
+                      uint32_t* status) {
   const long long t = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
   if (t >= n) return;
   const int y = targets[t];
   if ((y < 0 || y >= v) && status) atomicOr(status, A3PO_STATUS_TARGET_OUT_OF_RANGE);
-  if (row_mask && row_mask[t] == 0) {
+  // c = row of the partials: the row itself, or its place in the compact row space (-1: not computed)
+  const long long c = pos ? static_cast<long long>(pos[t]) : t;
+  if ((row_mask && row_mask[t] == 0) || c < 0) {
     logp[t] = 0.f;
     lse[t] = 0.f;
     if (entropy) entropy[t] = 0.f;
     return;
   }
   float m = -INFINITY;
-  for (int i = 0; i < splits; ++i) m = fmaxf(m, part[static_cast<long long>(i) * n + t].m);
+  for (int i = 0; i < splits; ++i) m = fmaxf(m, part[static_cast<long long>(i) * n + c].m);
   float s = 0.f, e = 0.f;
   for (int i = 0; i < splits; ++i) {
-    const SoftmaxPartial q = part[static_cast<long long>(i) * n + t];
+    const SoftmaxPartial q = part[static_cast<long long>(i) * n + c];
     const float scale = expf(q.m - m);
     s = fmaf(q.s, scale, s);
-    if (entropy) e = fmaf(part_ent[static_cast<long long>(i) * n + t], scale, e);
+    if (entropy) e = fmaf(part_ent[static_cast<long long>(i) * n + c], scale, e);
   }
   const float l = m + logf(s);
   lse[t] = l;
-  logp[t] = zy[t] - l;
+  logp[t] = zy[c] - l;
   if (entropy) entropy[t] = l - e / s;
 }
 
@@ -191,7 +194,7 @@ const char* a3po_kernel_name(int kernel_id) {
   static const char* names[kKernelIdCount] = {
       "loss_fwd", "loss_bwd", "loss_fwd_bwd", "loss_finalize", "mask_count", "mask_count_finalize",
       "expand_versions", "merge_partials", "lmhead_fwd_fp32pipe", "lmhead_dz_fp32pipe", "gemm_fp32pipe",
-      "gemm_tn<fwd_logsoftmax>", "gemm_tn<dz>", "gemm_tn<grad_hidden>", "gemm_tn<grad_w>", "transpose_bf16"};
+      "gemm_tn<fwd_logsoftmax>", "gemm_tn<dz>", "gemm_tn<grad_hidden>", "gemm_tn<grad_w>", "compact_rows"};
   return (kernel_id >= 0 && kernel_id < kKernelIdCount) ? names[kernel_id] : "?";
 }
 
@@ -244,10 +247,12 @@ size_t a3po_token_logprobs_min_workspace_bytes(int64_t N, int H, int V, a3po_dty
 
 size_t a3po_token_logprobs_workspace_bytes(int64_t N, int H, int V, a3po_dtype dt, int is_bwd) {
   if (N < 0 || H <= 0 || V <= 0) return 0;
-  if (!is_bwd) return a3po_token_logprobs_min_workspace_bytes(N, H, V, dt, 0);
+  // the recommended size adds room for the row compaction of the tensor-core path
+  const size_t compact = (dt == A3PO_BF16 && N > 0) ? compact_ws_bytes(N, H, is_bwd != 0) : 0;
+  if (!is_bwd) return a3po_token_logprobs_min_workspace_bytes(N, H, V, dt, 0) + compact;
   size_t a = simt_bwd_ws(clamp_chunk(kSimtChunkRows, N, kSimtTile), V);
   if (dt == A3PO_BF16) {
-    const size_t b = lmhead_tc_bwd_ws_bytes(clamp_chunk(kTcChunkRows, N, 128), N, H, V);
+    const size_t b = lmhead_tc_bwd_ws_bytes(clamp_chunk(kTcChunkRows, N, 128), N, H, V) + compact;
     if (b > a) a = b;
   }
   return a;
@@ -264,22 +269,36 @@ int a3po_token_logprobs_fwd(const void* hidden, const void* w, const int32_t* ta
   const bool tc = use_tc(dt, hidden, w, N, H, V);
   const int splits = tc ? lmhead_tc_fwd_splits(N, V) : simt_fwd_splits(N, V);
   if (ws_bytes < fwd_ws_for(N, splits)) return A3PO_ERR_WORKSPACE;
-  Arena arena(ws, ws_bytes);
+  // Masked rows are skipped, not computed: with a row mask and enough workspace the kept rows are
+  // gathered into a compact buffer and the kernels run on that (count stays on the device).
+  CompactBuffers cb;
+  bool compacted = false;
+  size_t ws_off = 0;
+  if (tc && row_mask && ws_bytes >= fwd_ws_for(N, splits) + compact_ws_bytes(N, H, false)) {
+    if (!compact_carve(ws, ws_bytes, N, H, false, &cb, &ws_off)) return A3PO_ERR_WORKSPACE;
+    compacted = true;
+  }
+  Arena arena(static_cast<char*>(ws) + ws_off, ws_bytes - ws_off);
   SoftmaxPartial* part = arena.take<SoftmaxPartial>(static_cast<size_t>(N) * splits);
   float* part_ent = arena.take<float>(static_cast<size_t>(N) * splits);
   float* zy = arena.take<float>(static_cast<size_t>(N));
   if (!arena.ok()) return A3PO_ERR_WORKSPACE;
   if (!entropy) part_ent = nullptr;
-  if (tc) {
-    A3PO_RETURN_IF(lmhead_fwd_tc(hidden, w, targets, N, H, V, inv_temperature, splits, part, part_ent, zy, status,
-                                 stream));
+  if (compacted) {
+    A3PO_RETURN_IF(compact_rows(hidden, H, targets, row_mask, nullptr, nullptr, N, cb, stream));
+    A3PO_RETURN_IF(lmhead_fwd_tc(cb.hidden_c, w, cb.targets_c, N, H, V, inv_temperature, splits, part, part_ent, zy,
+                                 cb.count, status, stream));
+  } else if (tc) {
+    A3PO_RETURN_IF(lmhead_fwd_tc(hidden, w, targets, N, H, V, inv_temperature, splits, part, part_ent, zy, nullptr,
+                                 status, stream));
   } else {
     A3PO_RETURN_IF(lmhead_fwd_simt(hidden, w, targets, N, H, V, dt, inv_temperature, splits, part, part_ent, zy,
                                    stream));
   }
   const unsigned blocks = static_cast<unsigned>((N + kMergeThreads - 1) / kMergeThreads);
   A3PO_LAUNCH(kKMergePartials, stream, (merge_partials_kernel<<<blocks, kMergeThreads, 0, stream>>>(
-                                           part, part_ent, zy, targets, row_mask, N, V, splits, logp, lse, entropy, status)));
+                                           part, part_ent, zy, targets, row_mask, compacted ? cb.pos : nullptr, N, V,
+                                           splits, logp, lse, entropy, status)));
   return after_launch();
 }
 
@@ -293,12 +312,27 @@ int a3po_token_logprobs_bwd(const void* hidden, const void* w, const int32_t* ta
   if (!ws || !aligned_to(ws, 256)) return A3PO_ERR_WORKSPACE;
   cudaStream_t stream = as_stream(stream_);
   if (use_tc(dt, hidden, w, N, H, V) && N > 0) {
-    // largest chunk (multiple of 128 rows) whose scratch fits the caller's buffer
+    // Rows with a zero upstream gradient (padding, clipped tokens) are skipped: with enough workspace
+    // the other rows are gathered into a compact buffer first (their count stays on the device).
+    CompactBuffers cb;
+    size_t ws_off = 0;
+    const bool compacted = ws_bytes >= compact_ws_bytes(N, H, true) + lmhead_tc_bwd_ws_bytes(128, N, H, V) &&
+                           compact_carve(ws, ws_bytes, N, H, true, &cb, &ws_off);
+    if (!compacted) ws_off = 0;
+    void* ws_rest = static_cast<char*>(ws) + ws_off;
+    const size_t rest_bytes = ws_bytes - ws_off;
+    // largest chunk (multiple of 128 rows) whose scratch fits what is left of the caller's buffer
     long long chunk = clamp_chunk(kTcChunkRows, N, 128);
-    while (chunk > 128 && lmhead_tc_bwd_ws_bytes(chunk, N, H, V) > ws_bytes) chunk -= 128;
-    if (lmhead_tc_bwd_ws_bytes(chunk, N, H, V) > ws_bytes) return A3PO_ERR_WORKSPACE;
-    return lmhead_bwd_tc(hidden, w, targets, lse, grad_logp, N, H, V, inv_temperature, grad_hidden, grad_w,
-                         accumulate_grad_w, ws, ws_bytes, chunk, status, stream);
+    while (chunk > 128 && lmhead_tc_bwd_ws_bytes(chunk, N, H, V) > rest_bytes) chunk -= 128;
+    if (lmhead_tc_bwd_ws_bytes(chunk, N, H, V) > rest_bytes) return A3PO_ERR_WORKSPACE;
+    if (!compacted)
+      return lmhead_bwd_tc(hidden, w, targets, lse, grad_logp, N, H, V, inv_temperature, grad_hidden, grad_w,
+                           accumulate_grad_w, ws_rest, rest_bytes, chunk, nullptr, status, stream);
+    A3PO_RETURN_IF(compact_rows(hidden, H, targets, nullptr, grad_logp, lse, N, cb, stream));
+    A3PO_RETURN_IF(lmhead_bwd_tc(cb.hidden_c, w, cb.targets_c, cb.lse_c, cb.g_c, N, H, V, inv_temperature,
+                                 cb.grad_hidden_c, grad_w, accumulate_grad_w, ws_rest, rest_bytes, chunk, cb.count,
+                                 status, stream));
+    return scatter_rows(cb.grad_hidden_c, H, cb.pos, N, grad_hidden, stream);
   }
   if (ws_bytes < simt_bwd_ws(kSimtTile, V)) return A3PO_ERR_WORKSPACE;
   long long chunk = clamp_chunk(kSimtChunkRows, N, kSimtTile);

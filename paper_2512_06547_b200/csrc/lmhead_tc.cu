@@ -53,6 +53,13 @@ struct ItemMap {
   int n_tiles;
   int splits;
   long long items;
+  // Optional device-side row count (compact row space): this launch covers rows
+  // [dyn_offset, dyn_offset + dyn_cap) of it and really has clamp(*dyn_rows - dyn_offset, 0, dyn_cap).
+  const int* dyn_rows;   // null: extents are the static ones above
+  int dyn_is_k;          // 0: the rows are the M extent; 1: the rows are the K extent
+  int zero_when_empty;   // dyn_is_k only: with no rows, store an all-zero output instead of doing nothing
+  long long dyn_offset;
+  long long dyn_cap;
 };
 
 struct Item {
@@ -379,8 +386,26 @@ __device__ __forceinline__ bool all_epilogue_threads(bool pred) {
 template <class Epi, bool A_MN, bool B_MN>
 __global__ void __launch_bounds__(kTcThreads, 1)
 gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-               const __grid_constant__ CUtensorMap map_c, ItemMap im, int k_blocks, typename Epi::Params ep,
-               uint32_t* status) {
+               const __grid_constant__ CUtensorMap map_c, ItemMap im_static, int k_blocks_static,
+               typename Epi::Params ep, uint32_t* status) {
+  // Work extents: static, or derived from the device-resident row count (identical in every thread).
+  ItemMap im = im_static;
+  int k_blocks = k_blocks_static;
+  bool zero_output = false;  // K extent is empty: the product is the zero matrix
+  if (im.dyn_rows != nullptr) {
+    long long rows = static_cast<long long>(*im.dyn_rows) - im.dyn_offset;
+    rows = rows < 0 ? 0 : (rows > im.dyn_cap ? im.dyn_cap : rows);
+    if (im.dyn_is_k) {
+      k_blocks = static_cast<int>((rows + BK - 1) / BK);
+      if (k_blocks == 0) {
+        if (im.zero_when_empty) zero_output = true;
+        else im.items = 0;
+      }
+    } else {
+      im.m_tiles = static_cast<int>((rows + BM - 1) / BM);
+      im.items = static_cast<long long>(im.m_tiles) * im.splits;
+    }
+  }
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* smem_a = smem;
@@ -422,7 +447,9 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   const uint32_t tmem_base = *tmem_slot;
 
   bool ok = true;
-  if (warp == 0) {
+  if (warp < 2 && zero_output) {
+    // nothing to load or multiply: the epilogue warps write zeros
+  } else if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (elect_one()) {
       int stage = 0;
@@ -509,21 +536,30 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       epi.begin(ep, static_cast<long long>(tile_row0) + row_in_tile);
       for (int nt = it.n_begin; nt < it.n_end && ok; ++nt) {
         // the four epilogue warps share named barriers further down: they must agree on giving up
-        ok = all_epilogue_threads(mbar_wait(&tmem_full_bar[acc], acc_phase, abort_flag));
-        if (!ok) break;
-        tcgen05_fence_after_sync();
+        if (!zero_output) {
+          ok = all_epilogue_threads(mbar_wait(&tmem_full_bar[acc], acc_phase, abort_flag));
+          if (!ok) break;
+          tcgen05_fence_after_sync();
+        }
         const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(acc * BN);
 #pragma unroll 1
         for (int c = 0; c < BN / kEpiChunk; ++c) {
           uint32_t r[kEpiChunk];
-          tmem_ld_32x32(taddr + static_cast<uint32_t>(c * kEpiChunk), r);
-          tmem_ld_wait();
+          if (!zero_output) {
+            tmem_ld_32x32(taddr + static_cast<uint32_t>(c * kEpiChunk), r);
+            tmem_ld_wait();
+          } else {
+#pragma unroll
+            for (int j = 0; j < kEpiChunk; ++j) r[j] = 0u;
+          }
           epi.chunk(ep, tile_row0, nt * BN + c * kEpiChunk, r, st);
         }
-        tcgen05_fence_before_sync();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&tmem_empty_bar[acc]);
-        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        if (!zero_output) {
+          tcgen05_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&tmem_empty_bar[acc]);
+          if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        }
       }
       if (ok) epi.end(ep, static_cast<long long>(tile_row0) + row_in_tile, it.split);
     }
@@ -570,9 +606,18 @@ int make_map(CUtensorMap* map, const Operand& op, bool mn_major, int tile_mn) {
 }
 
 // C[M, N] = sum_k A[m, k] B[n, k];  splits = 0 means one column tile per work item.
+// Device-resident row count for a launch (see ItemMap).
+struct DynRows {
+  const int* rows = nullptr;
+  int is_k = 0;
+  int zero_when_empty = 0;
+  long long offset = 0;
+  long long cap = 0;
+};
+
 template <class Epi, bool A_MN, bool B_MN>
-int launch_gemm(const Operand& a, const Operand& b, int splits, const typename Epi::Params& ep, uint32_t* status,
-                cudaStream_t stream) {
+int launch_gemm(const Operand& a, const Operand& b, int splits, const typename Epi::Params& ep, const DynRows& dyn,
+                uint32_t* status, cudaStream_t stream) {
   CUtensorMap map_a, map_b, map_c;
   A3PO_RETURN_IF(make_map(&map_a, a, A_MN, BM));
   A3PO_RETURN_IF(make_map(&map_b, b, B_MN, BN));
@@ -582,6 +627,11 @@ int launch_gemm(const Operand& a, const Operand& b, int splits, const typename E
   im.n_tiles = static_cast<int>((b.mn_extent + BN - 1) / BN);
   im.splits = splits > 0 ? splits : im.n_tiles;
   im.items = static_cast<long long>(im.m_tiles) * im.splits;
+  im.dyn_rows = dyn.rows;
+  im.dyn_is_k = dyn.is_k;
+  im.zero_when_empty = dyn.zero_when_empty;
+  im.dyn_offset = dyn.offset;
+  im.dyn_cap = dyn.cap;
   const int k_blocks = static_cast<int>((a.k_extent + BK - 1) / BK);
   auto kernel = gemm_tn_kernel<Epi, A_MN, B_MN>;
   if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemBytes)) !=
@@ -633,16 +683,19 @@ int lmhead_tc_fwd_splits(long long n, int v) {
 }
 
 int lmhead_fwd_tc(const void* hidden, const void* w, const int32_t* targets, long long n, int h, int v, float inv_t,
-                  int splits, SoftmaxPartial* part, float* part_ent, float* zy, uint32_t* status,
+                  int splits, SoftmaxPartial* part, float* part_ent, float* zy, const int* dyn_rows, uint32_t* status,
                   cudaStream_t stream) {
   const Operand a{hidden, n, h, h};
   const Operand b{w, v, h, h};
+  DynRows dyn;
+  dyn.rows = dyn_rows;
+  dyn.cap = n;
   if (part_ent) {
     FwdEpilogue<true>::Params p{targets, n, v, inv_t * kLog2e, inv_t, part, part_ent, zy};
-    return launch_gemm<FwdEpilogue<true>, false, false>(a, b, splits, p, status, stream);
+    return launch_gemm<FwdEpilogue<true>, false, false>(a, b, splits, p, dyn, status, stream);
   }
   FwdEpilogue<false>::Params p{targets, n, v, inv_t * kLog2e, inv_t, part, nullptr, zy};
-  return launch_gemm<FwdEpilogue<false>, false, false>(a, b, splits, p, status, stream);
+  return launch_gemm<FwdEpilogue<false>, false, false>(a, b, splits, p, dyn, status, stream);
 }
 
 size_t lmhead_tc_bwd_ws_bytes(long long chunk_rows, long long /*n*/, int /*h*/, int v) {
@@ -651,8 +704,8 @@ size_t lmhead_tc_bwd_ws_bytes(long long chunk_rows, long long /*n*/, int /*h*/, 
 
 int lmhead_bwd_tc(const void* hidden_, const void* w_, const int32_t* targets, const float* lse,
                   const float* grad_logp, long long n, int h, int v, float inv_t, void* grad_hidden_, float* grad_w,
-                  int accumulate, void* ws, size_t ws_bytes, long long chunk_rows, uint32_t* status,
-                  cudaStream_t stream) {
+                  int accumulate, void* ws, size_t ws_bytes, long long chunk_rows, const int* dyn_rows,
+                  uint32_t* status, cudaStream_t stream) {
   const __nv_bfloat16* hidden = static_cast<const __nv_bfloat16*>(hidden_);
   const __nv_bfloat16* w = static_cast<const __nv_bfloat16*>(w_);
   __nv_bfloat16* grad_hidden = static_cast<__nv_bfloat16*>(grad_hidden_);
@@ -666,16 +719,23 @@ int lmhead_bwd_tc(const void* hidden_, const void* w_, const int32_t* targets, c
     const __nv_bfloat16* hid_c = hidden + r0 * h;
     // dz[t, v] for this chunk of rows, from recomputed logits:  A = hidden (K-major), B = W (K-major)
     DzEpilogue::Params dp{targets, lse, grad_logp, r0, r1, v, vpad, inv_t * kLog2e, inv_t, dz};
+    DynRows dyn_m;  // dz and grad_hidden: the rows are the M extent
+    dyn_m.rows = dyn_rows;
+    dyn_m.offset = r0;
+    dyn_m.cap = nc;
+    DynRows dyn_k = dyn_m;  // grad_w: the rows are the K extent
+    dyn_k.is_k = 1;
+    dyn_k.zero_when_empty = (r0 == 0 && !accumulate) ? 1 : 0;
     A3PO_RETURN_IF((launch_gemm<DzEpilogue, false, false>(Operand{hid_c, nc, h, h}, Operand{w, v, h, h}, 0, dp,
-                                                          status, stream)));
+                                                          dyn_m, status, stream)));
     // grad_hidden[t, j] = sum_v dz[t, v] W[v, j]:  A = dz (K = v contiguous), B = W read N-major
     StoreBf16Epilogue::Params hp{grad_hidden + r0 * h, h, nc, h};
     A3PO_RETURN_IF((launch_gemm<StoreBf16Epilogue, false, true>(Operand{dz, nc, v, vpad}, Operand{w, h, v, h}, 0, hp,
-                                                                status, stream)));
+                                                                dyn_m, status, stream)));
     // grad_w[v, j] (+)= sum_t dz[t, v] hidden[t, j]:  A = dz read M-major, B = hidden read N-major (K = t)
     StoreF32Epilogue::Params wp{grad_w, h, v, h, (accumulate || r0 > 0) ? 1 : 0};
     A3PO_RETURN_IF((launch_gemm<StoreF32Epilogue, true, true>(Operand{dz, v, nc, vpad}, Operand{hid_c, h, nc, h}, 0,
-                                                              wp, status, stream)));
+                                                              wp, dyn_k, status, stream)));
   }
   return A3PO_OK;
 }
