@@ -353,7 +353,8 @@ def run_ours(args):
         entry = {"kernel": name, "launches": cnt, "ms_total": round(ms, 4), "share": round(ms / kernel_total, 4)}
         if name.startswith("gemm_tn"):
             entry["rows"] = rows_of.get(name, n)
-            entry["tflops"] = round(2.0 * entry["rows"] * v * h * cnt / (ms * 1e-3) / 1e12, 1)
+            # a step may split a contraction over several launches (row chunks): flops are per step
+            entry["tflops"] = round(2.0 * entry["rows"] * v * h * args.steps / (ms * 1e-3) / 1e12, 1)
         kernels.append(entry)
     dom = kernels[0]
     sustained = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
@@ -365,7 +366,7 @@ def run_ours(args):
                     "peak_burst": peaks["bf16_tflops"], "frac_of_burst": round(achieved / peaks["bf16_tflops"], 4),
                     "frac_of_nominal_2250": round(achieved / 2250.0, 4),
                     "all_gemm_tn_tflops": round(
-                        sum(2.0 * k["rows"] * v * h * k["launches"] for k in kernels if k["kernel"].startswith("gemm_tn")) /
+                        sum(2.0 * k["rows"] * v * h * args.steps for k in kernels if k["kernel"].startswith("gemm_tn")) /
                         (sum(k["ms_total"] for k in kernels if k["kernel"].startswith("gemm_tn")) * 1e-3) / 1e12, 1)}
     else:
         roofline = {"bound": "hbm", "kernel": dom["kernel"], "achieved": None, "peak": peaks["hbm_gbs"],

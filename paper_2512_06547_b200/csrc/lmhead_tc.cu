@@ -18,6 +18,7 @@
 // Every mbarrier wait is bounded; on expiry the CTA raises A3PO_STATUS_WAIT_TIMEOUT in the
 // caller's status word, releases its TMEM and exits.
 
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 
@@ -52,6 +53,7 @@ struct ItemMap {
   int m_tiles;
   int n_tiles;
   int splits;
+  int group_m;  // row tiles per rasterisation group
   long long items;
   // Optional device-side row count (compact row space): this launch covers rows
   // [dyn_offset, dyn_offset + dyn_cap) of it and really has clamp(*dyn_rows - dyn_offset, 0, dyn_cap).
@@ -70,6 +72,7 @@ struct Item {
 };
 
 __device__ __forceinline__ Item decode_item(const ItemMap& im, long long i) {
+  const int kGroupM = im.group_m;
   const long long per_group = static_cast<long long>(kGroupM) * im.splits;
   const int full_groups = im.m_tiles / kGroupM;
   Item it;
@@ -606,6 +609,14 @@ int make_map(CUtensorMap* map, const Operand& op, bool mn_major, int tile_mn) {
 }
 
 // C[M, N] = sum_k A[m, k] B[n, k];  splits = 0 means one column tile per work item.
+// Tuning overrides read from the environment (positive integers); used for sweeps, not needed in normal use.
+int tuning_override(const char* name, int fallback) {
+  const char* e = std::getenv(name);
+  if (!e) return fallback;
+  const int v = std::atoi(e);
+  return v > 0 ? v : fallback;
+}
+
 // Device-resident row count for a launch (see ItemMap).
 struct DynRows {
   const int* rows = nullptr;
@@ -627,6 +638,7 @@ int launch_gemm(const Operand& a, const Operand& b, int splits, const typename E
   im.n_tiles = static_cast<int>((b.mn_extent + BN - 1) / BN);
   im.splits = splits > 0 ? splits : im.n_tiles;
   im.items = static_cast<long long>(im.m_tiles) * im.splits;
+  im.group_m = tuning_override("A3PO_GROUP_M", kGroupM);
   im.dyn_rows = dyn.rows;
   im.dyn_is_k = dyn.is_k;
   im.zero_when_empty = dyn.zero_when_empty;
@@ -668,6 +680,8 @@ int lmhead_tc_fwd_splits(long long n, int v) {
   if (m_tiles <= 0) return 1;
   int sms = sm_count();
   if (sms <= 0) sms = 148;
+  const int forced = tuning_override("A3PO_FWD_SPLITS", 0);
+  if (forced > 0) return forced < n_tiles ? (forced < 64 ? forced : 64) : n_tiles;
   const int s_max = n_tiles < 64 ? n_tiles : 64;
   int s_min = s_max < 8 ? s_max : 8;  // several splits in flight keep the row-tile working set inside L2
   int best = s_min;

@@ -145,3 +145,37 @@ def test_empty_batch():
 def test_full_vocab_sub_batch_1p5b():
     """Full-size V and H of the 1.5B-shaped config on a sub-batch of rows (all outputs)."""
     _check_fwd_bwd(384, 1536, workloads.QWEN_VOCAB, "bf16", seed=61, want_entropy=False)
+
+
+def test_masked_and_zero_gradient_rows_are_skipped_consistently():
+    """Row compaction: any pattern of masked rows (forward) or zero upstream gradients (backward), including
+    none and all of them, gives the same numbers as the oracle; grad_w is exactly zero / untouched when no row
+    takes part."""
+    n, h, v = 700, 256, 2000
+    hidden, w, targets, g = _problem(n, h, v, "bf16", 71)
+    hn, wn, tn = to_np64(hidden), to_np64(w), targets.cpu().numpy()
+    rng = np.random.default_rng(72)
+    for keep_frac in (0.0, 0.03, 0.5, 1.0):
+        mask_np = (rng.random(n) < keep_frac).astype(np.uint8)
+        mask = torch.from_numpy(mask_np).to(DEV)
+        logp, lse, _, status = gpu_fwd(hidden, w, targets, row_mask=mask)
+        assert status == 0
+        logp_ref, lse_ref = orc.token_logprobs_fwd(hn, wn, tn, row_mask=mask_np)
+        assert np.max(np.abs(logp.cpu().numpy() - logp_ref), initial=0.0) <= LOGP_TOL_BF16
+        assert np.max(np.abs(lse.cpu().numpy() - lse_ref), initial=0.0) <= LOGP_TOL_BF16
+        assert not logp.cpu().numpy()[mask_np == 0].any()
+        # backward with the upstream gradient restricted to the kept rows
+        g_np = g.cpu().numpy() * mask_np
+        full_lse = torch.from_numpy(orc.token_logprobs_fwd(hn, wn, tn)[1].astype(np.float32)).to(DEV)
+        gh, gw, status = gpu_bwd(hidden, w, targets, full_lse, torch.from_numpy(g_np).to(DEV))
+        assert status == 0
+        gh_ref, gw_ref = orc.token_logprobs_bwd(hn, wn, tn, g_np.astype(np.float64))
+        if g_np.any():
+            assert rel_fro(to_np64(gh), gh_ref) <= GRAD_FRO_RTOL and rel_fro(to_np64(gw), gw_ref) <= GRAD_FRO_RTOL
+        else:
+            assert not gh.float().abs().sum().item() and not gw.abs().sum().item()     # overwritten with zeros
+            base = torch.randn(v, h, device=DEV)
+            _, acc, _ = gpu_bwd(hidden, w, targets, full_lse, torch.zeros(n, device=DEV), grad_w=base.clone(),
+                                accumulate=True)
+            assert torch.equal(acc, base)                                              # accumulate: untouched
+        assert not to_np64(gh)[g_np == 0].any()
