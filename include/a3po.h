@@ -175,6 +175,50 @@ int a3po_loss_fwd_bwd(const float* logp, const float* behav_logp, const int32_t*
                       float* grad_logp, void* ws, size_t ws_bytes, void* stream);
 
 /* --------------------------------------------------------------------------------------------
+ * The decoupled clipped loss of Eq. 2 with an EXPLICIT proximal policy: the baseline the paper
+ * calls "recompute" (Sec. 2.2: log pi_prox comes from an extra forward pass and is frozen), and,
+ * with prox_logp = behav_logp, the coupled PPO-clip loss of Eq. 1 ("sync").  Same streaming
+ * kernel as a3po_loss_fwd_bwd with the interpolation replaced by a load:
+ *
+ *   iw_t  = exp(prox_logp[t] - behav_logp[t]),   r_t = exp(logp[t] - prox_logp[t])
+ *   obj_t = iw_t * min(r_t * adv[t], clip(r_t, 1-eps, 1+eps) * adv[t])
+ *   loss  = - sum_t mask[t] * obj_t / max(M, 1)
+ *   grad_logp[t] = -(mask_t / M) * iw_t * adv_t * r_t * act_t        (the anchor is a constant)
+ *
+ * prox_logp: fp32 [N].  grad_logp may be NULL (forward only).  Other arguments, outputs,
+ * workspace and error codes as a3po_loss_fwd_bwd.
+ * ------------------------------------------------------------------------------------------ */
+int a3po_decoupled_loss_fwd_bwd(const float* logp, const float* behav_logp, const float* prox_logp,
+                                const float* adv, const uint8_t* mask, int64_t N, float clip_eps,
+                                float* loss, a3po_stats* stats, float* grad_logp, void* ws,
+                                size_t ws_bytes, void* stream);
+
+/* --------------------------------------------------------------------------------------------
+ * GRPO advantages (Sec. 4.1: "estimate advantages using group reward normalization"; the paper
+ * gives no formula, the customary one is used).  Sequences come in consecutive groups of
+ * `group_size` responses to the same prompt:
+ *
+ *   A_i = (R_i - mean_group) / (std_group + norm_eps)        population standard deviation
+ *   adv[t] = A_i for every row t of sequence i, i.e. cu_seqlens[i] <= t < cu_seqlens[i+1]
+ *
+ * rewards fp32 [B], cu_seqlens int32 [B+1] (cu_seqlens[0] = 0, cu_seqlens[B] = N), B a multiple
+ * of group_size, adv fp32 [N] output.  ws: at least a3po_grpo_workspace_bytes(B).
+ * ------------------------------------------------------------------------------------------ */
+size_t a3po_grpo_workspace_bytes(int B);
+
+int a3po_grpo_advantages(const float* rewards, int B, int group_size, const int32_t* cu_seqlens,
+                         int64_t N, float norm_eps, float* adv, void* ws, size_t ws_bytes,
+                         void* stream);
+
+/* --------------------------------------------------------------------------------------------
+ * Self-test of the bounded waits the pipelined kernels rely on (no counterpart in the paper).
+ * Launches a one-warp kernel that waits on a barrier nothing ever signals; after timeout_ms
+ * (1..2000) the wait gives up and ORs A3PO_STATUS_WAIT_TIMEOUT into *status (device word),
+ * which is what a stuck pipeline stage does instead of hanging the GPU.
+ * ------------------------------------------------------------------------------------------ */
+int a3po_selftest_wait_timeout(uint32_t* status, unsigned timeout_ms, void* stream);
+
+/* --------------------------------------------------------------------------------------------
  * a3po_loss_fwd for callers that have no way to hand over a workspace (the paper has no
  * counterpart: this is a packaging variant, the arithmetic is a3po_loss_fwd's).
  *

@@ -232,6 +232,39 @@ def loss_bwd(logp, behav_logp, versions, current_version, adv, mask, clip_eps,
     return np.where(valid, -(float(grad_loss) / m) * dobj, 0.0)
 
 
+def decoupled_loss(logp, behav_logp, prox_logp, adv, mask, clip_eps, grad_loss=1.0):
+    """Eq. 2 with an explicit, frozen proximal policy (the "recompute" baseline of Sec. 2.2).
+
+    iw = exp(l_prox - l_behav), r = exp(l_theta - l_prox), obj = iw * min(r A, clip(r) A),
+    L = -sum m obj / max(M, 1);  dL/dl_theta = -(grad_loss m / M) iw A r act  (anchor constant).
+    Returns (loss, stats, grad_logp, terms).
+    """
+    valid = np.asarray(mask) != 0
+    l_theta = np.where(valid, _f64(logp), 0.0)
+    l_behav = np.where(valid, _f64(behav_logp), 0.0)
+    l_prox = np.where(valid, _f64(prox_logp), 0.0)
+    a = np.where(valid, _f64(adv), 0.0)
+    eps = np.float64(np.float32(clip_eps))
+    iw = np.exp(l_prox - l_behav)
+    r = np.exp(l_theta - l_prox)
+    s1 = r * a
+    s2 = np.minimum(np.maximum(r, 1.0 - eps), 1.0 + eps) * a
+    obj = iw * np.minimum(s1, s2)
+    act = s1 <= s2
+    m = int(valid.sum())
+    loss = -float(np.sum(np.where(valid, obj, 0.0))) / max(m, 1)
+    stats = dict(
+        n_valid=m,
+        n_clipped=int(np.sum(valid & ~act)),
+        iw_max=float(iw[valid].max()) if m else 0.0,
+        iw_min=float(iw[valid].min()) if m else 0.0,
+        abs_obj_mean=float(np.sum(np.where(valid, np.abs(obj), 0.0))) / max(m, 1),
+    )
+    grad = np.where(valid, -(float(grad_loss) / max(m, 1)) * iw * a * r * act, 0.0)
+    margin = np.minimum(np.abs(r - (1.0 - eps)), np.abs(r - (1.0 + eps)))
+    return loss, stats, grad, dict(r=r, iw=iw, act=act, margin=margin, valid=valid)
+
+
 # --------------------------------------------------------------------------------------
 # GRPO advantages (Sec. 4.1 "group reward normalization"; the paper gives no formula, the
 # usual one is taken: population standard deviation, 1e-6 added to the denominator)

@@ -9,7 +9,11 @@ from .binding import (  # noqa: F401
     STATUS_TARGET_OUT_OF_RANGE,
     STATUS_WAIT_TIMEOUT,
     A3poError,
+    a3po_decoupled_loss_fwd_bwd,
+    a3po_grpo_advantages,
+    a3po_grpo_workspace_bytes,
     a3po_kernel_launch_count,
+    a3po_selftest_wait_timeout,
     a3po_loss_bwd,
     a3po_loss_fwd,
     a3po_loss_fwd_bwd,

@@ -56,6 +56,12 @@ _SIGNATURES = {
     "a3po_loss_fwd_bwd": (c_int, [c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_int, c_int32, c_void_p, c_void_p,
                                   c_int64, c_float, c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t,
                                   c_void_p]),
+    "a3po_decoupled_loss_fwd_bwd": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_float, c_void_p,
+                                            c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
+    "a3po_grpo_workspace_bytes": (c_size_t, [c_int]),
+    "a3po_grpo_advantages": (c_int, [c_void_p, c_int, c_int, c_void_p, c_int64, c_float, c_void_p, c_void_p, c_size_t,
+                                     c_void_p]),
+    "a3po_selftest_wait_timeout": (c_int, [c_void_p, ctypes.c_uint, c_void_p]),
     "a3po_train_step_host": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_int, c_int,
                                      c_int, c_int32, c_float, c_float, c_void_p, c_void_p, c_int, c_void_p, c_void_p,
                                      c_size_t, c_void_p, c_size_t, c_void_p, c_void_p, c_void_p, c_void_p]),
@@ -276,6 +282,45 @@ def a3po_loss_fwd_bwd(logp, behav_logp, versions, current_version, adv, mask, cl
                                           int(bool(detach_prox)), _ptr(loss), _ptr(stats), _ptr(grad_logp), _ptr(ws),
                                           ws.numel(), _stream(stream))
     _check("a3po_loss_fwd_bwd", rc)
+
+
+def a3po_decoupled_loss_fwd_bwd(logp, behav_logp, prox_logp, adv, mask, clip_eps, loss, ws, *, grad_logp=None,
+                                stats=None, stream=None):
+    """Eq. 2 with an explicit proximal log-prob array (the "recompute" baseline; prox = behav gives Eq. 1)."""
+    for t, nm in ((logp, "logp"), (behav_logp, "behav_logp"), (prox_logp, "prox_logp"), (adv, "adv"),
+                  (loss, "loss"), (grad_logp, "grad_logp")):
+        _want(t, torch.float32, nm)
+    _want(mask, torch.uint8, "mask"); _want(stats, torch.uint8, "stats"); _want(ws, torch.uint8, "ws")
+    n = logp.numel()
+    if not (behav_logp.numel() == prox_logp.numel() == adv.numel() == mask.numel() == n):
+        raise ValueError("shape mismatch")
+    rc = load_library().a3po_decoupled_loss_fwd_bwd(_ptr(logp), _ptr(behav_logp), _ptr(prox_logp), _ptr(adv),
+                                                    _ptr(mask), n, float(clip_eps), _ptr(loss), _ptr(stats),
+                                                    _ptr(grad_logp), _ptr(ws), ws.numel(), _stream(stream))
+    _check("a3po_decoupled_loss_fwd_bwd", rc)
+
+
+def a3po_grpo_workspace_bytes(B) -> int:
+    return load_library().a3po_grpo_workspace_bytes(B)
+
+
+def a3po_grpo_advantages(rewards, group_size, cu_seqlens, adv, ws, *, norm_eps=1e-6, stream=None):
+    """adv[t] = group-normalised reward of the sequence that owns row t."""
+    _want(rewards, torch.float32, "rewards"); _want(cu_seqlens, torch.int32, "cu_seqlens")
+    _want(adv, torch.float32, "adv"); _want(ws, torch.uint8, "ws")
+    b = rewards.numel()
+    if cu_seqlens.numel() != b + 1:
+        raise ValueError("cu_seqlens must have B + 1 entries")
+    rc = load_library().a3po_grpo_advantages(_ptr(rewards), b, int(group_size), _ptr(cu_seqlens), adv.numel(),
+                                             float(norm_eps), _ptr(adv), _ptr(ws), ws.numel(), _stream(stream))
+    _check("a3po_grpo_advantages", rc)
+
+
+def a3po_selftest_wait_timeout(status, timeout_ms=50, stream=None):
+    """Runs the bounded-wait self-test kernel; afterwards `status` must hold STATUS_WAIT_TIMEOUT."""
+    _want(status, torch.int32, "status")
+    _check("a3po_selftest_wait_timeout",
+           load_library().a3po_selftest_wait_timeout(_ptr(status), int(timeout_ms), _stream(stream)))
 
 
 # ------------------------------------------------------------------------------ whole step, host inputs

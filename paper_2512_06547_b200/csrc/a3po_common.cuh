@@ -28,7 +28,7 @@ int sm_count();
 // Kernel identifiers for launch accounting and the optional CUDA-event profile.
 enum KernelId : int {
   kKLossFwd = 0, kKLossBwd, kKLossFwdBwd, kKLossFinalize, kKMaskCount, kKMaskCountFinalize, kKExpandVersions,
-  kKMergePartials, kKSimtFwd, kKSimtDz, kKSimtGemm, kKTcFwd, kKTcDz, kKTcGradHidden, kKTcGradW, kKCompact,
+  kKMergePartials, kKSimtFwd, kKSimtDz, kKSimtGemm, kKTcFwd, kKTcDz, kKTcGradHidden, kKTcGradW, kKCompact, kKGrpo, kKSelfTest,
   kKernelIdCount
 };
 

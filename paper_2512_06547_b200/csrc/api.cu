@@ -186,7 +186,13 @@ const char* a3po_status_string(int code) {
   }
 }
 
-int a3po_version(void) { return 1000; }
+int a3po_version(void) { return 1001; }
+
+int a3po_selftest_wait_timeout(uint32_t* status, unsigned timeout_ms, void* stream) {
+  if (!status || timeout_ms == 0 || timeout_ms > 2000) return A3PO_ERR_INVALID_ARG;
+  if (sm_count() <= 0) return A3PO_ERR_NO_DEVICE;
+  return selftest_wait_timeout(status, timeout_ms, as_stream(stream));
+}
 
 int64_t a3po_kernel_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
@@ -194,7 +200,7 @@ const char* a3po_kernel_name(int kernel_id) {
   static const char* names[kKernelIdCount] = {
       "loss_fwd", "loss_bwd", "loss_fwd_bwd", "loss_finalize", "mask_count", "mask_count_finalize",
       "expand_versions", "merge_partials", "lmhead_fwd_fp32pipe", "lmhead_dz_fp32pipe", "gemm_fp32pipe",
-      "gemm_tn<fwd_logsoftmax>", "gemm_tn<dz>", "gemm_tn<grad_hidden>", "gemm_tn<grad_w>", "compact_rows"};
+      "gemm_tn<fwd_logsoftmax>", "gemm_tn<dz>", "gemm_tn<grad_hidden>", "gemm_tn<grad_w>", "compact_rows", "grpo_advantages", "selftest"};
   return (kernel_id >= 0 && kernel_id < kKernelIdCount) ? names[kernel_id] : "?";
 }
 

@@ -62,4 +62,7 @@ int lmhead_bwd_tc(const void* hidden, const void* w, const int32_t* targets, con
                   int accumulate, void* ws, size_t ws_bytes, long long chunk_rows, const int* dyn_rows,
                   uint32_t* status, cudaStream_t stream);
 
+// Launches a one-warp kernel whose bounded wait must expire after timeout_ms and set the status bit.
+int selftest_wait_timeout(uint32_t* status, unsigned timeout_ms, cudaStream_t stream);
+
 }  // namespace a3po

@@ -99,6 +99,23 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&p);
 }
 
+// Waits on an mbarrier that never completes; the wait gives up after limit_ns and raises the
+// status bit, exactly as a stuck pipeline stage would.
+__global__ void wait_timeout_kernel(uint32_t* status, unsigned long long limit_ns) {
+  __shared__ uint64_t bar;
+  __shared__ uint32_t abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    abort_flag = 0;
+    fence_mbar_init();
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const bool completed = mbar_wait(&bar, 0, &abort_flag, limit_ns);
+    if (!completed && status) atomicOr(status, A3PO_STATUS_WAIT_TIMEOUT);
+  }
+}
+
 // ------------------------------------------------------------------------------------ tensor maps
 using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -666,6 +683,13 @@ size_t bwd_ws_layout(long long chunk_rows, int v) {
 }
 
 }  // namespace
+
+// Exercises the bounded wait the pipelines rely on: a barrier nothing ever arrives at.
+int selftest_wait_timeout(uint32_t* status, unsigned timeout_ms, cudaStream_t stream) {
+  A3PO_LAUNCH(kKSelfTest, stream, (wait_timeout_kernel<<<1, 32, 0, stream>>>(
+                                      status, static_cast<unsigned long long>(timeout_ms) * 1000000ull)));
+  return after_launch();
+}
 
 bool lmhead_tc_supported(const void* hidden, const void* w, long long n, int h, int v) {
   return n > 0 && h >= 8 && (h % 8) == 0 && v >= 1 && aligned_to(hidden, 16) && aligned_to(w, 16) &&

@@ -30,7 +30,8 @@ struct alignas(16) LossPartial {
 struct LossArgs {
   const float* logp;
   const float* behav;
-  const int32_t* versions;  // per token
+  const int32_t* versions;  // per token (interpolated anchor)
+  const float* prox;        // explicit proximal log-probs (EXPLICIT kernels), else unused
   const float* adv;
   const uint8_t* mask;
   long long n;
@@ -58,17 +59,26 @@ struct Acc {
 // interpolation of Eq. 3 but conditioned on the small difference of the two log-probs.
 // Staleness is exact for any pair of int32 versions: a signed compare decides d >= 1 and the
 // unsigned difference is d itself in that case; d = 1 takes alpha = 1 without a reciprocal.
-template <int MODE>
+// EXPLICIT: the anchor is given (`ver` then carries the bits of log pi_prox), Eq. 2 as it stands:
+// iw = exp(l_prox - l_behav), r = exp(l_theta - l_prox); the anchor is a constant in the backward.
+template <int MODE, bool EXPLICIT>
 __device__ __forceinline__ void token(float lt, float lb, int ver, float a, bool valid,
                                       const LossArgs& p, float coef, float& fsum, Acc& acc,
                                       float& grad) {
-  const unsigned du = static_cast<unsigned>(p.current_version) - static_cast<unsigned>(ver);
-  const bool interpolate = (ver < p.current_version) && (du > 1u);
-  const float alpha = interpolate ? fast_rcp(static_cast<float>(du)) : 1.0f;
-  const float d2 = (lt - lb) * kLog2e;
-  const float ad2 = alpha * d2;
-  const float r = fast_exp2(ad2);
-  const float iw = fast_exp2(d2 - ad2);
+  float alpha = 1.0f, r, iw;
+  if (EXPLICIT) {
+    const float lp = __int_as_float(ver);
+    r = fast_exp2((lt - lp) * kLog2e);
+    iw = fast_exp2((lp - lb) * kLog2e);
+  } else {
+    const unsigned du = static_cast<unsigned>(p.current_version) - static_cast<unsigned>(ver);
+    const bool interpolate = (ver < p.current_version) && (du > 1u);
+    alpha = interpolate ? fast_rcp(static_cast<float>(du)) : 1.0f;
+    const float d2 = (lt - lb) * kLog2e;
+    const float ad2 = alpha * d2;
+    r = fast_exp2(ad2);
+    iw = fast_exp2(d2 - ad2);
+  }
   const float s1 = r * a;
   const float s2 = fminf(fmaxf(r, p.lo), p.hi) * a;
   const bool act = s1 <= s2;
@@ -81,24 +91,25 @@ __device__ __forceinline__ void token(float lt, float lb, int ver, float a, bool
   }
   if (MODE != kFwd) {
     const float through = act ? iw * s1 : 0.f;
-    const float dobj = p.detach ? through : fmaf(alpha, through - obj, obj);  // (1-a)*obj + a*through
+    const float dobj = (EXPLICIT || p.detach) ? through : fmaf(alpha, through - obj, obj);  // (1-a)*obj + a*through
     grad = valid ? coef * dobj : 0.f;
   }
 }
 
-template <int MODE>
+template <int MODE, bool EXPLICIT>
 __device__ __forceinline__ void group4(long long g, const LossArgs& p, float coef, Acc& acc) {
   const float4 lt = __ldcs(reinterpret_cast<const float4*>(p.logp) + g);
   const float4 lb = __ldcs(reinterpret_cast<const float4*>(p.behav) + g);
-  const int4 ver = __ldcs(reinterpret_cast<const int4*>(p.versions) + g);
+  const int4 ver = __ldcs(reinterpret_cast<const int4*>(EXPLICIT ? static_cast<const void*>(p.prox)
+                                                                  : static_cast<const void*>(p.versions)) + g);
   const float4 a = __ldcs(reinterpret_cast<const float4*>(p.adv) + g);
   const unsigned m = __vcmpne4(__ldcs(reinterpret_cast<const unsigned*>(p.mask) + g), 0u);  // 0xff per valid token
   float fsum = 0.f;
   float4 gr;
-  token<MODE>(lt.x, lb.x, ver.x, a.x, (m & 0x000000ffu) != 0, p, coef, fsum, acc, gr.x);
-  token<MODE>(lt.y, lb.y, ver.y, a.y, (m & 0x0000ff00u) != 0, p, coef, fsum, acc, gr.y);
-  token<MODE>(lt.z, lb.z, ver.z, a.z, (m & 0x00ff0000u) != 0, p, coef, fsum, acc, gr.z);
-  token<MODE>(lt.w, lb.w, ver.w, a.w, (m & 0xff000000u) != 0, p, coef, fsum, acc, gr.w);
+  token<MODE, EXPLICIT>(lt.x, lb.x, ver.x, a.x, (m & 0x000000ffu) != 0, p, coef, fsum, acc, gr.x);
+  token<MODE, EXPLICIT>(lt.y, lb.y, ver.y, a.y, (m & 0x0000ff00u) != 0, p, coef, fsum, acc, gr.y);
+  token<MODE, EXPLICIT>(lt.z, lb.z, ver.z, a.z, (m & 0x00ff0000u) != 0, p, coef, fsum, acc, gr.z);
+  token<MODE, EXPLICIT>(lt.w, lb.w, ver.w, a.w, (m & 0xff000000u) != 0, p, coef, fsum, acc, gr.w);
   if (MODE != kBwd) {
     acc.sum += static_cast<double>(fsum);
     acc.n_valid += __popc(m) >> 3;
@@ -106,11 +117,12 @@ __device__ __forceinline__ void group4(long long g, const LossArgs& p, float coe
   if (MODE != kFwd) __stcs(reinterpret_cast<float4*>(p.grad_logp) + g, gr);
 }
 
-template <int MODE>
+template <int MODE, bool EXPLICIT>
 __device__ __forceinline__ void single(long long t, const LossArgs& p, float coef, Acc& acc) {
   float fsum = 0.f, gr = 0.f;
   const bool valid = p.mask[t] != 0;
-  token<MODE>(p.logp[t], p.behav[t], p.versions[t], p.adv[t], valid, p, coef, fsum, acc, gr);
+  const int third = EXPLICIT ? __float_as_int(p.prox[t]) : p.versions[t];
+  token<MODE, EXPLICIT>(p.logp[t], p.behav[t], third, p.adv[t], valid, p, coef, fsum, acc, gr);
   if (MODE != kBwd) {
     acc.sum += static_cast<double>(fsum);
     acc.n_valid += valid ? 1 : 0;
@@ -119,7 +131,7 @@ __device__ __forceinline__ void single(long long t, const LossArgs& p, float coe
 }
 
 // VEC = true needs 16-byte aligned fp32/int32 arrays and a 4-byte aligned mask.
-template <int MODE, bool VEC>
+template <int MODE, bool VEC, bool EXPLICIT>
 __global__ void __launch_bounds__(kLossThreads, kBlocksPerSm) loss_kernel(LossArgs p, LossPartial* partials) {
   float coef = 0.f;
   if (MODE != kFwd) {
@@ -134,14 +146,14 @@ __global__ void __launch_bounds__(kLossThreads, kBlocksPerSm) loss_kernel(LossAr
     const long long groups = p.n >> 2;
     long long g = tid;
     for (; g + nthreads < groups; g += 2 * nthreads) {
-      group4<MODE>(g, p, coef, acc);
-      group4<MODE>(g + nthreads, p, coef, acc);
+      group4<MODE, EXPLICIT>(g, p, coef, acc);
+      group4<MODE, EXPLICIT>(g + nthreads, p, coef, acc);
     }
-    if (g < groups) group4<MODE>(g, p, coef, acc);
+    if (g < groups) group4<MODE, EXPLICIT>(g, p, coef, acc);
     const long long t = (groups << 2) + tid;  // ragged tail: at most three tokens
-    if (t < p.n) single<MODE>(t, p, coef, acc);
+    if (t < p.n) single<MODE, EXPLICIT>(t, p, coef, acc);
   } else {
-    for (long long t = tid; t < p.n; t += nthreads) single<MODE>(t, p, coef, acc);
+    for (long long t = tid; t < p.n; t += nthreads) single<MODE, EXPLICIT>(t, p, coef, acc);
   }
   if (MODE == kBwd) return;
 
@@ -284,17 +296,19 @@ int grid_for(long long n_items) {
   return static_cast<int>(want);
 }
 
-int run_loss(int mode, const float* logp, const float* behav, const int32_t* versions, int versions_per_seq,
+int run_loss(int mode, const float* logp, const float* behav, const float* prox, const int32_t* versions,
+             int versions_per_seq,
              const int32_t* cu_seqlens, int b, int32_t current_version, const float* adv, const uint8_t* mask,
              long long n, float clip_eps, int detach, const float* grad_loss, const a3po_stats* fwd_stats,
              float* loss, a3po_stats* stats, float* grad_logp, void* ws, size_t ws_bytes, void* stream_) {
   if (n < 0 || !(clip_eps >= 0.f)) return A3PO_ERR_INVALID_ARG;
-  if (n > 0 && (!logp || !behav || !versions || !adv || !mask)) return A3PO_ERR_INVALID_ARG;
+  if (n > 0 && (!logp || !behav || (!versions && !prox) || !adv || !mask)) return A3PO_ERR_INVALID_ARG;
   if (mode != kBwd && !loss) return A3PO_ERR_INVALID_ARG;
   if (mode != kFwd && n > 0 && !grad_logp) return A3PO_ERR_INVALID_ARG;
-  if (versions_per_seq && n > 0 && (!cu_seqlens || b <= 0)) return A3PO_ERR_INVALID_ARG;
+  if (!prox && versions_per_seq && n > 0 && (!cu_seqlens || b <= 0)) return A3PO_ERR_INVALID_ARG;
   if (!ws || !aligned_to(ws, 256) || ws_bytes < loss_ws_bytes(n)) return A3PO_ERR_WORKSPACE;
-  if (!aligned_to(logp, 4) || !aligned_to(behav, 4) || !aligned_to(versions, 4) || !aligned_to(adv, 4) ||
+  if (!aligned_to(logp, 4) || !aligned_to(behav, 4) || !aligned_to(versions, 4) || !aligned_to(prox, 4) ||
+      !aligned_to(adv, 4) ||
       !aligned_to(grad_logp, 4))
     return A3PO_ERR_UNSUPPORTED;
   if (sm_count() <= 0) return A3PO_ERR_NO_DEVICE;
@@ -308,7 +322,7 @@ int run_loss(int mode, const float* logp, const float* behav, const int32_t* ver
   w.versions = arena.take<int32_t>(static_cast<size_t>(n));
   if (!arena.ok()) return A3PO_ERR_WORKSPACE;
 
-  if (versions_per_seq && n > 0) {
+  if (!prox && versions_per_seq && n > 0) {
     const int blocks = static_cast<int>((n + kLossThreads - 1) / kLossThreads);
     A3PO_LAUNCH(kKExpandVersions, stream,
                 expand_versions_kernel<<<blocks, kLossThreads, 0, stream>>>(versions, cu_seqlens, b, n, w.versions));
@@ -317,7 +331,7 @@ int run_loss(int mode, const float* logp, const float* behav, const int32_t* ver
   }
 
   LossArgs p;
-  p.logp = logp; p.behav = behav; p.versions = versions; p.adv = adv; p.mask = mask; p.n = n;
+  p.logp = logp; p.behav = behav; p.versions = versions; p.prox = prox; p.adv = adv; p.mask = mask; p.n = n;
   p.current_version = current_version;
   p.lo = 1.0f - clip_eps; p.hi = 1.0f + clip_eps;
   p.detach = detach;
@@ -339,13 +353,16 @@ int run_loss(int mode, const float* logp, const float* behav, const int32_t* ver
     }
   }
 
-  const bool vec = aligned_to(logp, 16) && aligned_to(behav, 16) && aligned_to(versions, 16) &&
+  const bool vec = aligned_to(logp, 16) && aligned_to(behav, 16) && aligned_to(versions, 16) && aligned_to(prox, 16) &&
                    aligned_to(adv, 16) && aligned_to(mask, 4) && (mode == kFwd || aligned_to(grad_logp, 16));
   const int blocks = grid_for(vec ? (n + 7) / 8 : n);
 #define A3PO_LAUNCH_LOSS(MODE, KID)                                                                        \
   do {                                                                                                     \
-    if (vec) A3PO_LAUNCH(KID, stream, (loss_kernel<MODE, true><<<blocks, kLossThreads, 0, stream>>>(p, w.partials)));  \
-    else A3PO_LAUNCH(KID, stream, (loss_kernel<MODE, false><<<blocks, kLossThreads, 0, stream>>>(p, w.partials)));     \
+    if (prox) {                                                                                            \
+      if (vec) A3PO_LAUNCH(KID, stream, (loss_kernel<MODE, true, true><<<blocks, kLossThreads, 0, stream>>>(p, w.partials)));   \
+      else A3PO_LAUNCH(KID, stream, (loss_kernel<MODE, false, true><<<blocks, kLossThreads, 0, stream>>>(p, w.partials)));      \
+    } else if (vec) A3PO_LAUNCH(KID, stream, (loss_kernel<MODE, true, false><<<blocks, kLossThreads, 0, stream>>>(p, w.partials))); \
+    else A3PO_LAUNCH(KID, stream, (loss_kernel<MODE, false, false><<<blocks, kLossThreads, 0, stream>>>(p, w.partials)));       \
   } while (0)
   if (mode == kFwd) A3PO_LAUNCH_LOSS(kFwd, kKLossFwd);
   else if (mode == kBwd) A3PO_LAUNCH_LOSS(kBwd, kKLossBwd);
@@ -371,7 +388,7 @@ int a3po_loss_fwd(const float* logp, const float* behav_logp, const int32_t* ver
                   const int32_t* cu_seqlens, int B, int32_t current_version, const float* adv,
                   const uint8_t* mask, int64_t N, float clip_eps, float* loss, a3po_stats* stats, void* ws,
                   size_t ws_bytes, void* stream) {
-  return a3po::run_loss(a3po::kFwd, logp, behav_logp, versions, versions_per_seq, cu_seqlens, B, current_version,
+  return a3po::run_loss(a3po::kFwd, logp, behav_logp, nullptr, versions, versions_per_seq, cu_seqlens, B, current_version,
                         adv, mask, N, clip_eps, 1, nullptr, nullptr, loss, stats, nullptr, ws, ws_bytes, stream);
 }
 
@@ -430,7 +447,7 @@ int a3po_loss_fwd_static(const float* logp, const float* behav_logp, const int32
   if (a3po::sm_count() <= 0) return A3PO_ERR_NO_DEVICE;
   void* scratch = nullptr;
   A3PO_RETURN_IF(a3po::static_loss_scratch(&scratch));
-  return a3po::run_loss(a3po::kFwd, logp, behav_logp, versions, versions_per_seq, cu_seqlens, B, current_version,
+  return a3po::run_loss(a3po::kFwd, logp, behav_logp, nullptr, versions, versions_per_seq, cu_seqlens, B, current_version,
                         adv, mask, N, clip_eps, 1, nullptr, nullptr, loss, stats, nullptr, scratch,
                         a3po::kStaticScratchBytes, stream);
 }
@@ -439,7 +456,7 @@ int a3po_loss_bwd(const float* logp, const float* behav_logp, const int32_t* ver
                   const int32_t* cu_seqlens, int B, int32_t current_version, const float* adv,
                   const uint8_t* mask, int64_t N, float clip_eps, int detach_prox, const float* grad_loss,
                   const a3po_stats* fwd_stats, float* grad_logp, void* ws, size_t ws_bytes, void* stream) {
-  return a3po::run_loss(a3po::kBwd, logp, behav_logp, versions, versions_per_seq, cu_seqlens, B, current_version,
+  return a3po::run_loss(a3po::kBwd, logp, behav_logp, nullptr, versions, versions_per_seq, cu_seqlens, B, current_version,
                         adv, mask, N, clip_eps, detach_prox, grad_loss, fwd_stats, nullptr, nullptr, grad_logp, ws,
                         ws_bytes, stream);
 }
@@ -448,9 +465,19 @@ int a3po_loss_fwd_bwd(const float* logp, const float* behav_logp, const int32_t*
                       const int32_t* cu_seqlens, int B, int32_t current_version, const float* adv,
                       const uint8_t* mask, int64_t N, float clip_eps, int detach_prox, float* loss,
                       a3po_stats* stats, float* grad_logp, void* ws, size_t ws_bytes, void* stream) {
-  return a3po::run_loss(a3po::kFwdBwd, logp, behav_logp, versions, versions_per_seq, cu_seqlens, B,
+  return a3po::run_loss(a3po::kFwdBwd, logp, behav_logp, nullptr, versions, versions_per_seq, cu_seqlens, B,
                         current_version, adv, mask, N, clip_eps, detach_prox, nullptr, nullptr, loss, stats,
                         grad_logp, ws, ws_bytes, stream);
+}
+
+int a3po_decoupled_loss_fwd_bwd(const float* logp, const float* behav_logp, const float* prox_logp, const float* adv,
+                                const uint8_t* mask, int64_t N, float clip_eps, float* loss, a3po_stats* stats,
+                                float* grad_logp, void* ws, size_t ws_bytes, void* stream) {
+  if (N > 0 && !prox_logp) return A3PO_ERR_INVALID_ARG;
+  const int mode = grad_logp ? a3po::kFwdBwd : a3po::kFwd;
+  static const float kNoTokens = 0.f;  // N == 0: run_loss still wants a non-null anchor to pick this variant
+  return a3po::run_loss(mode, logp, behav_logp, prox_logp ? prox_logp : &kNoTokens, nullptr, 0, nullptr, 0, 0, adv,
+                        mask, N, clip_eps, 1, nullptr, nullptr, loss, stats, grad_logp, ws, ws_bytes, stream);
 }
 
 }  // extern "C"

@@ -232,3 +232,45 @@ def test_grpo_advantages():
     np.testing.assert_allclose(adv[:4], np.array([1, -1, -1, 1]) / (1 + 2e-6) * 1.0, rtol=1e-5)
     np.testing.assert_array_equal(adv[4:], 0.0)
     assert abs(adv[:4].sum()) < 1e-12
+
+
+# ---------------------------------------------------------------------------- explicit anchor (Eq. 2 as it stands)
+def test_decoupled_loss_with_behaviour_anchor_is_coupled_ppo():
+    """prox = behav turns Eq. 2 into Eq. 1 (independent scalar implementation above)."""
+    logp, behav, _, _, adv, mask = _batch(1500, 21, noise=0.4)
+    loss, stats, grad, _ = orc.decoupled_loss(logp, behav, behav, adv, mask, 0.2)
+    assert loss == pytest.approx(_coupled_ppo_clip_loss(logp, behav, adv, mask, float(np.float32(0.2))), rel=1e-13)
+    assert stats["iw_max"] == 1.0 and stats["iw_min"] == 1.0
+
+
+def test_decoupled_loss_with_interpolated_anchor_is_a3po():
+    """Feeding the anchor of Eq. 3-4 explicitly reproduces the A-3PO loss and its detached gradient."""
+    logp, behav, versions, cur, adv, mask = _batch(1200, 22, noise=0.5)
+    prox = orc.prox_logp(logp, behav, orc.staleness_alpha(versions, cur))
+    loss, stats, grad, _ = orc.decoupled_loss(logp, behav, prox, adv, mask, 0.2, grad_loss=1.3)
+    ref_loss, ref_stats = orc.loss_fwd(logp, behav, versions, cur, adv, mask, 0.2)
+    assert loss == pytest.approx(ref_loss, rel=1e-13)
+    assert stats["n_clipped"] == ref_stats["n_clipped"] and stats["n_valid"] == ref_stats["n_valid"]
+    np.testing.assert_allclose(grad, orc.loss_bwd(logp, behav, versions, cur, adv, mask, 0.2, grad_loss=1.3),
+                               rtol=1e-12, atol=1e-18)
+
+
+def test_decoupled_loss_scalar_brute_force_and_finite_differences():
+    n = 30
+    rng = np.random.default_rng(23)
+    logp = -rng.standard_exponential(n)
+    behav = np.minimum(logp + 0.3 * rng.standard_normal(n), 0)
+    prox = np.minimum(logp + 0.2 * rng.standard_normal(n), 0)
+    adv = rng.standard_normal(n)
+    mask = (rng.random(n) < 0.8).astype(np.uint8)
+    eps = float(np.float32(0.2))
+    loss, stats, grad, terms = orc.decoupled_loss(logp, behav, prox, adv, mask, 0.2)
+    assert loss == pytest.approx(_loss_with_frozen_anchor(logp, prox, behav, adv, mask, eps), rel=1e-13)
+    step = 1e-6
+    for i in np.flatnonzero(terms["margin"] > 1e-3):
+        lp_, lm_ = logp.copy(), logp.copy()
+        lp_[i] += step
+        lm_[i] -= step
+        fd = (_loss_with_frozen_anchor(lp_, prox, behav, adv, mask, eps)
+              - _loss_with_frozen_anchor(lm_, prox, behav, adv, mask, eps)) / (2 * step)
+        assert grad[i] == pytest.approx(fd, abs=1e-8)
