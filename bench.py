@@ -257,11 +257,16 @@ def run_ours(args):
     behav = to_dev(behav_host)
 
     def step():
-        a3po.a3po_token_logprobs_fwd(wl.hidden, wl.w, targets, logp, lse, ws, row_mask=mask, status=status)
-        a3po.a3po_loss_fwd_bwd(logp, behav, versions, wl.current_version, adv, mask, wl.clip_eps, loss, grad_logp,
-                               ws, stats=stats)
-        a3po.a3po_token_logprobs_bwd(wl.hidden, wl.w, targets, lse, grad_logp, grad_hidden, grad_w, ws,
-                                     status=status)
+        if args.separate_calls:     # the three ABI calls one after the other: the backward recomputes the logits
+            a3po.a3po_token_logprobs_fwd(wl.hidden, wl.w, targets, logp, lse, ws, row_mask=mask, status=status)
+            a3po.a3po_loss_fwd_bwd(logp, behav, versions, wl.current_version, adv, mask, wl.clip_eps, loss,
+                                   grad_logp, ws, stats=stats)
+            a3po.a3po_token_logprobs_bwd(wl.hidden, wl.w, targets, lse, grad_logp, grad_hidden, grad_w, ws,
+                                         status=status)
+        else:                       # one call; the backward reuses the logits the forward kept in the workspace
+            a3po.a3po_train_step(wl.hidden, wl.w, targets, behav, versions, wl.current_version, adv, mask,
+                                 wl.clip_eps, logp, lse, grad_logp, loss, grad_hidden, grad_w, ws, stats=stats,
+                                 status=status)
 
     sampler = ClockSampler(local_rank)
     if rank == 0:
@@ -345,9 +350,11 @@ def run_ours(args):
     # clipped tokens are skipped by the library, so they are not counted as work).
     fwd_rows = n_valid
     bwd_rows = int((grad_logp != 0).sum().item())
-    rows_of = {"gemm_tn<fwd_logsoftmax>": fwd_rows, "gemm_tn<dz>": bwd_rows, "gemm_tn<grad_hidden>": bwd_rows,
-               "gemm_tn<grad_w>": bwd_rows}
-    step_flops = 2.0 * v * h * (fwd_rows + 3 * bwd_rows)
+    rows_of = {"gemm_tn<fwd_logsoftmax>": fwd_rows, "gemm_tn<fwd_logsoftmax+keep_logits>": fwd_rows,
+               "gemm_tn<dz>": bwd_rows, "gemm_tn<grad_hidden>": bwd_rows, "gemm_tn<grad_w>": bwd_rows}
+    # contractions actually executed per step: forward + (dz recompute unless the logits were kept) + two gradients
+    recomputes = any(name == "gemm_tn<dz>" for name in agg)
+    step_flops = 2.0 * v * h * (fwd_rows + (3 if recomputes else 2) * bwd_rows)
     kernels = []
     for name, (cnt, ms) in sorted(agg.items(), key=lambda kv: -kv[1][1]):
         entry = {"kernel": name, "launches": cnt, "ms_total": round(ms, 4), "share": round(ms / kernel_total, 4)}
@@ -502,6 +509,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--small", action="store_true",
                     help="same shapes with 4 sequences only (a profiler-sized case; not a benchmark number)")
+    ap.add_argument("--separate-calls", action="store_true",
+                    help="time fwd / loss / bwd as three ABI calls (backward recomputes the logits) instead of "
+                         "a3po_train_step")
     args = ap.parse_args()
     if args.workload == "loss_sweep":
         run_loss_sweep(args)

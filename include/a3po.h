@@ -263,6 +263,29 @@ int a3po_loss_fwd_static(const float* logp, const float* behav_logp, const int32
  * d_ws a3po_train_step_workspace_bytes(N,H,V,dt).  h_loss (float) and h_stats are host outputs,
  * valid after the caller synchronises `stream`.
  * ------------------------------------------------------------------------------------------ */
+/* --------------------------------------------------------------------------------------------
+ * One whole training-step pass with every buffer on the device (no counterpart in the paper):
+ *   logp, lse   = token_logprobs_fwd(hidden, w, targets, row_mask = mask)
+ *   loss, stats, grad_logp = loss_fwd_bwd(logp, behav_logp, versions (per token), ...)   detach_prox = 1
+ *   grad_hidden, grad_w    = token_logprobs_bwd(..., lse, grad_logp)
+ * with the same results as the three calls.  Given a workspace of
+ * a3po_train_step_workspace_bytes(...) and bf16 inputs, the forward keeps its logits (fp16, shifted
+ * by a per-row, per-256-column reference so that the entries that matter are stored accurately;
+ * rows with mask != 0 only) and the backward builds dz from them in one streaming pass instead of
+ * recomputing the LM head: 6 N V H flops per step instead of 8 N V H.  The kept logits live in the
+ * workspace only (N_valid x V x 2 bytes).  With a smaller workspace (at least
+ * a3po_train_step_min_workspace_bytes) the three calls are made as they are.
+ * logp, lse, grad_logp: fp32 [N] outputs.  Other arguments as in the individual calls.
+ * ------------------------------------------------------------------------------------------ */
+size_t a3po_train_step_min_workspace_bytes(int64_t N, int H, int V, a3po_dtype dt);
+
+int a3po_train_step(const void* hidden, const int32_t* targets, const float* behav_logp,
+                    const int32_t* versions, const float* adv, const uint8_t* mask, int64_t N, int H,
+                    int V, a3po_dtype dt, int32_t current_version, float clip_eps,
+                    float inv_temperature, const void* w, float* grad_w, int accumulate_grad_w,
+                    void* grad_hidden, float* logp, float* lse, float* grad_logp, float* loss,
+                    a3po_stats* stats, void* ws, size_t ws_bytes, uint32_t* status, void* stream);
+
 size_t a3po_train_step_stage_bytes(int64_t N, int H, a3po_dtype dt);
 size_t a3po_train_step_workspace_bytes(int64_t N, int H, int V, a3po_dtype dt);
 

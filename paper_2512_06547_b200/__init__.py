@@ -25,7 +25,9 @@ from .binding import (  # noqa: F401
     a3po_token_logprobs_fwd,
     a3po_token_logprobs_min_workspace_bytes,
     a3po_token_logprobs_workspace_bytes,
+    a3po_train_step,
     a3po_train_step_host,
+    a3po_train_step_min_workspace_bytes,
     a3po_train_step_stage_bytes,
     a3po_train_step_workspace_bytes,
     a3po_version,

@@ -62,6 +62,10 @@ _SIGNATURES = {
     "a3po_grpo_advantages": (c_int, [c_void_p, c_int, c_int, c_void_p, c_int64, c_float, c_void_p, c_void_p, c_size_t,
                                      c_void_p]),
     "a3po_selftest_wait_timeout": (c_int, [c_void_p, ctypes.c_uint, c_void_p]),
+    "a3po_train_step_min_workspace_bytes": (c_size_t, [c_int64, c_int, c_int, c_int]),
+    "a3po_train_step": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_int, c_int, c_int,
+                                c_int32, c_float, c_float, c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_void_p,
+                                c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p, c_void_p]),
     "a3po_train_step_host": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_int, c_int,
                                      c_int, c_int32, c_float, c_float, c_void_p, c_void_p, c_int, c_void_p, c_void_p,
                                      c_size_t, c_void_p, c_size_t, c_void_p, c_void_p, c_void_p, c_void_p]),
@@ -321,6 +325,38 @@ def a3po_selftest_wait_timeout(status, timeout_ms=50, stream=None):
     _want(status, torch.int32, "status")
     _check("a3po_selftest_wait_timeout",
            load_library().a3po_selftest_wait_timeout(_ptr(status), int(timeout_ms), _stream(stream)))
+
+
+# ------------------------------------------------------------------------------ whole step, device inputs
+def a3po_train_step_min_workspace_bytes(N, H, V, dt) -> int:
+    return load_library().a3po_train_step_min_workspace_bytes(N, H, V, dt)
+
+
+def a3po_train_step(hidden, w, targets, behav_logp, versions, current_version, adv, mask, clip_eps, logp, lse,
+                    grad_logp, loss, grad_hidden, grad_w, ws, *, stats=None, accumulate_grad_w=False,
+                    inv_temperature=1.0, status=None, stream=None):
+    """token_logprobs_fwd -> loss_fwd_bwd -> token_logprobs_bwd in one call; with the recommended workspace the
+    backward reuses logits kept by the forward instead of recomputing them."""
+    dt = _dtype_code(hidden)
+    _want(hidden, hidden.dtype, "hidden"); _want(w, hidden.dtype, "w"); _want(grad_hidden, hidden.dtype, "grad_hidden")
+    _want(targets, torch.int32, "targets"); _want(versions, torch.int32, "versions"); _want(mask, torch.uint8, "mask")
+    for t, nm in ((behav_logp, "behav_logp"), (adv, "adv"), (logp, "logp"), (lse, "lse"), (grad_logp, "grad_logp"),
+                  (loss, "loss"), (grad_w, "grad_w")):
+        _want(t, torch.float32, nm)
+    _want(stats, torch.uint8, "stats"); _want(status, torch.int32, "status"); _want(ws, torch.uint8, "ws")
+    n, h = hidden.shape
+    v = w.shape[0]
+    if w.shape[1] != h or grad_w.shape != w.shape or grad_hidden.shape != hidden.shape:
+        raise ValueError("shape mismatch")
+    for t in (targets, behav_logp, versions, adv, mask, logp, lse, grad_logp):
+        if t.numel() != n:
+            raise ValueError("per-token arrays must have N entries")
+    rc = load_library().a3po_train_step(
+        _ptr(hidden), _ptr(targets), _ptr(behav_logp), _ptr(versions), _ptr(adv), _ptr(mask), n, h, v, dt,
+        int(current_version), float(clip_eps), float(inv_temperature), _ptr(w), _ptr(grad_w),
+        int(bool(accumulate_grad_w)), _ptr(grad_hidden), _ptr(logp), _ptr(lse), _ptr(grad_logp), _ptr(loss),
+        _ptr(stats), _ptr(ws), ws.numel(), _ptr(status), _stream(stream))
+    _check("a3po_train_step", rc)
 
 
 # ------------------------------------------------------------------------------ whole step, host inputs

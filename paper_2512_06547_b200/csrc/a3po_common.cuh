@@ -3,6 +3,7 @@
 
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <stdint.h>
 #include <atomic>
 
@@ -28,7 +29,8 @@ int sm_count();
 // Kernel identifiers for launch accounting and the optional CUDA-event profile.
 enum KernelId : int {
   kKLossFwd = 0, kKLossBwd, kKLossFwdBwd, kKLossFinalize, kKMaskCount, kKMaskCountFinalize, kKExpandVersions,
-  kKMergePartials, kKSimtFwd, kKSimtDz, kKSimtGemm, kKTcFwd, kKTcDz, kKTcGradHidden, kKTcGradW, kKCompact, kKGrpo, kKSelfTest,
+  kKMergePartials, kKSimtFwd, kKSimtDz, kKSimtGemm, kKTcFwd, kKTcDz, kKTcGradHidden, kKTcGradW, kKCompact, kKGrpo,
+  kKSelfTest, kKTcFwdSave, kKDzSaved,
   kKernelIdCount
 };
 

@@ -133,10 +133,12 @@ size_t fwd_ws_for(long long n, int splits) {
          round_up(rows * sizeof(float), 256) + 256;
 }
 
-bool force_simt() {
-  const char* e = std::getenv("A3PO_FORCE_SIMT");
+bool env_flag(const char* name) {
+  const char* e = std::getenv(name);
   return e && e[0] == '1';
 }
+
+bool force_simt() { return env_flag("A3PO_FORCE_SIMT"); }
 
 bool use_tc(a3po_dtype dt, const void* hidden, const void* w, long long n, int h, int v) {
   return dt == A3PO_BF16 && !force_simt() && lmhead_tc_supported(hidden, w, n, h, v);
@@ -200,7 +202,8 @@ const char* a3po_kernel_name(int kernel_id) {
   static const char* names[kKernelIdCount] = {
       "loss_fwd", "loss_bwd", "loss_fwd_bwd", "loss_finalize", "mask_count", "mask_count_finalize",
       "expand_versions", "merge_partials", "lmhead_fwd_fp32pipe", "lmhead_dz_fp32pipe", "gemm_fp32pipe",
-      "gemm_tn<fwd_logsoftmax>", "gemm_tn<dz>", "gemm_tn<grad_hidden>", "gemm_tn<grad_w>", "compact_rows", "grpo_advantages", "selftest"};
+      "gemm_tn<fwd_logsoftmax>", "gemm_tn<dz>", "gemm_tn<grad_hidden>", "gemm_tn<grad_w>", "compact_rows", "grpo_advantages", "selftest",
+      "gemm_tn<fwd_logsoftmax+keep_logits>", "dz_from_kept_logits"};
   return (kernel_id >= 0 && kernel_id < kKernelIdCount) ? names[kernel_id] : "?";
 }
 
@@ -382,13 +385,113 @@ size_t a3po_train_step_stage_bytes(int64_t N, int H, a3po_dtype dt) {
   return stage_layout(N, H, dt).total;
 }
 
+namespace {
+// Workspace of the step that keeps the forward's logits (fp16, shifted) for the backward.
+struct SavedStepLayout {
+  size_t fwd_compact, bwd_compact, partials, saved, dz, loss, total;
+  int splits;
+};
+SavedStepLayout saved_step_layout(long long n, int h, int v) {
+  SavedStepLayout s;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = round_up(off + bytes, 256); return o; };
+  const long long cap = compact_capacity(n);
+  s.splits = lmhead_tc_fwd_splits(n, v);
+  s.fwd_compact = take(compact_ws_bytes(n, h, false));
+  s.bwd_compact = take(compact_ws_bytes(n, h, true));
+  s.partials = take(fwd_ws_for(n, s.splits));
+  s.saved = take(lmhead_tc_saved_logits_bytes(n, v));
+  s.dz = take(lmhead_tc_bwd_ws_bytes(cap, n, h, v));
+  s.loss = take(a3po_loss_workspace_bytes(n));
+  s.total = off;
+  return s;
+}
+}  // namespace
+
+size_t a3po_train_step_min_workspace_bytes(int64_t N, int H, int V, a3po_dtype dt) {
+  if (N < 0 || H <= 0 || V <= 0) return 0;
+  size_t a = a3po_token_logprobs_min_workspace_bytes(N, H, V, dt, 0);
+  const size_t b = a3po_token_logprobs_min_workspace_bytes(N, H, V, dt, 1);
+  const size_t c = a3po_loss_workspace_bytes(N);
+  if (b > a) a = b;
+  if (c > a) a = c;
+  return a;
+}
+
 size_t a3po_train_step_workspace_bytes(int64_t N, int H, int V, a3po_dtype dt) {
+  if (N < 0 || H <= 0 || V <= 0) return 0;
   size_t a = a3po_token_logprobs_workspace_bytes(N, H, V, dt, 0);
   const size_t b = a3po_token_logprobs_workspace_bytes(N, H, V, dt, 1);
   const size_t c = a3po_loss_workspace_bytes(N);
   if (b > a) a = b;
   if (c > a) a = c;
+  if (dt == A3PO_BF16 && N > 0) {
+    const size_t d = saved_step_layout(N, H, V).total;
+    if (d > a) a = d;
+  }
   return a;
+}
+
+int a3po_train_step(const void* hidden, const int32_t* targets, const float* behav_logp, const int32_t* versions,
+                    const float* adv, const uint8_t* mask, int64_t N, int H, int V, a3po_dtype dt,
+                    int32_t current_version, float clip_eps, float inv_temperature, const void* w, float* grad_w,
+                    int accumulate_grad_w, void* grad_hidden, float* logp, float* lse, float* grad_logp, float* loss,
+                    a3po_stats* stats, void* ws, size_t ws_bytes, uint32_t* status, void* stream_) {
+  A3PO_RETURN_IF(check_lmhead_args(hidden, w, targets, N, H, V, dt, inv_temperature));
+  if (!grad_w || !loss || (N > 0 && (!behav_logp || !versions || !adv || !mask || !grad_hidden || !logp || !lse ||
+                                      !grad_logp)))
+    return A3PO_ERR_INVALID_ARG;
+  if (!ws || !aligned_to(ws, 256)) return A3PO_ERR_WORKSPACE;
+  cudaStream_t stream = as_stream(stream_);
+
+  const bool keep_logits = N > 0 && use_tc(dt, hidden, w, N, H, V) && !env_flag("A3PO_NO_SAVED_LOGITS") &&
+                           ws_bytes >= saved_step_layout(N, H, V).total && aligned_to(grad_hidden, 16) &&
+                           aligned_to(grad_w, 16);
+  if (!keep_logits) {
+    // three independent calls; the backward recomputes the logits chunk by chunk
+    A3PO_RETURN_IF(a3po_token_logprobs_fwd(hidden, w, targets, mask, N, H, V, dt, inv_temperature, logp, lse, nullptr,
+                                           ws, ws_bytes, status, stream_));
+    A3PO_RETURN_IF(a3po_loss_fwd_bwd(logp, behav_logp, versions, 0, nullptr, 0, current_version, adv, mask, N,
+                                     clip_eps, 1, loss, stats, grad_logp, ws, ws_bytes, stream_));
+    return a3po_token_logprobs_bwd(hidden, w, targets, lse, grad_logp, N, H, V, dt, inv_temperature, grad_hidden,
+                                   grad_w, accumulate_grad_w, ws, ws_bytes, status, stream_);
+  }
+
+  // ---- forward on the rows with mask != 0, keeping shifted fp16 logits and their per-tile references
+  const SavedStepLayout lay = saved_step_layout(N, H, V);
+  char* base = static_cast<char*>(ws);
+  CompactBuffers fwd_cb, bwd_cb;
+  size_t used = 0;
+  if (!compact_carve(base + lay.fwd_compact, compact_ws_bytes(N, H, false), N, H, false, &fwd_cb, &used) ||
+      !compact_carve(base + lay.bwd_compact, compact_ws_bytes(N, H, true), N, H, true, &bwd_cb, &used))
+    return A3PO_ERR_WORKSPACE;
+  Arena arena(base + lay.partials, fwd_ws_for(N, lay.splits));
+  SoftmaxPartial* part = arena.take<SoftmaxPartial>(static_cast<size_t>(N) * lay.splits);
+  arena.take<float>(static_cast<size_t>(N) * lay.splits);  // entropy partials: unused here, same layout
+  float* zy = arena.take<float>(static_cast<size_t>(N));
+  if (!arena.ok()) return A3PO_ERR_WORKSPACE;
+  void* saved = base + lay.saved;
+  void* dz = base + lay.dz;
+
+  A3PO_RETURN_IF(compact_rows(hidden, H, targets, mask, nullptr, nullptr, N, fwd_cb, stream));
+  A3PO_RETURN_IF(lmhead_fwd_save_tc(fwd_cb.hidden_c, w, fwd_cb.targets_c, N, H, V, inv_temperature, lay.splits, part,
+                                    zy, saved, fwd_cb.count, status, stream));
+  {
+    const unsigned blocks = static_cast<unsigned>((N + kMergeThreads - 1) / kMergeThreads);
+    A3PO_LAUNCH(kKMergePartials, stream, (merge_partials_kernel<<<blocks, kMergeThreads, 0, stream>>>(
+                                             part, nullptr, zy, targets, mask, fwd_cb.pos, N, V, lay.splits, logp,
+                                             lse, nullptr, status)));
+    A3PO_RETURN_IF(after_launch());
+  }
+  // ---- loss and dL/dlogp on every token
+  A3PO_RETURN_IF(a3po_loss_fwd_bwd(logp, behav_logp, versions, 0, nullptr, 0, current_version, adv, mask, N, clip_eps,
+                                   1, loss, stats, grad_logp, base + lay.loss, a3po_loss_workspace_bytes(N), stream_));
+  // ---- backward on the rows with a non-zero upstream gradient: dz from the kept logits, two contractions
+  A3PO_RETURN_IF(compact_rows(hidden, H, targets, nullptr, grad_logp, lse, N, bwd_cb, stream));
+  A3PO_RETURN_IF(dz_from_saved(saved, N, V, fwd_cb.pos, bwd_cb, inv_temperature, dz, stream));
+  A3PO_RETURN_IF(lmhead_bwd_from_dz_tc(bwd_cb.hidden_c, w, dz, N, H, V, bwd_cb.grad_hidden_c, grad_w,
+                                       accumulate_grad_w, bwd_cb.count, status, stream));
+  return scatter_rows(bwd_cb.grad_hidden_c, H, bwd_cb.pos, N, grad_hidden, stream);
 }
 
 int a3po_train_step_host(const void* h_hidden, const int32_t* h_targets, const float* h_behav_logp,
@@ -429,13 +532,9 @@ int a3po_train_step_host(const void* h_hidden, const int32_t* h_targets, const f
   float* loss = reinterpret_cast<float*>(base + s.loss);
   a3po_stats* stats = reinterpret_cast<a3po_stats*>(base + s.stats);
 
-  A3PO_RETURN_IF(a3po_token_logprobs_fwd(hidden, d_w, targets, mask, N, H, V, dt, inv_temperature, logp, lse,
-                                         nullptr, d_ws, ws_bytes, d_status, stream_));
-  A3PO_RETURN_IF(a3po_loss_fwd_bwd(logp, behav, versions, 0, nullptr, 0, current_version, adv, mask, N, clip_eps, 1,
-                                   loss, stats, grad_logp, d_ws, ws_bytes, stream_));
-  A3PO_RETURN_IF(a3po_token_logprobs_bwd(hidden, d_w, targets, lse, grad_logp, N, H, V, dt, inv_temperature,
-                                         d_grad_hidden, d_grad_w, accumulate_grad_w, d_ws, ws_bytes, d_status,
-                                         stream_));
+  A3PO_RETURN_IF(a3po_train_step(hidden, targets, behav, versions, adv, mask, N, H, V, dt, current_version, clip_eps,
+                                 inv_temperature, d_w, d_grad_w, accumulate_grad_w, d_grad_hidden, logp, lse,
+                                 grad_logp, loss, stats, d_ws, ws_bytes, d_status, stream_));
   if (cudaMemcpyAsync(h_loss, loss, sizeof(float), cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
       (h_stats && cudaMemcpyAsync(h_stats, stats, sizeof(a3po_stats), cudaMemcpyDeviceToHost, stream) != cudaSuccess)) {
     cudaGetLastError();

@@ -62,6 +62,21 @@ int lmhead_bwd_tc(const void* hidden, const void* w, const int32_t* targets, con
                   int accumulate, void* ws, size_t ws_bytes, long long chunk_rows, const int* dyn_rows,
                   uint32_t* status, cudaStream_t stream);
 
+// ---- backward without recomputation (lmhead_tc.cu, saved_logits.cu) ----
+// The saving forward keeps, for n rows, u[n, v^8] (fp16: z log2(e)/T minus a per-(row, 256-column tile)
+// reference) followed by ref[n, tiles] (fp32) in one buffer of lmhead_tc_saved_logits_bytes(n, v) bytes.
+size_t lmhead_tc_saved_logits_bytes(long long n, int v);
+int lmhead_fwd_save_tc(const void* hidden, const void* w, const int32_t* targets, long long n, int h, int v,
+                       float inv_t, int splits, SoftmaxPartial* part, float* zy, void* saved, const int* dyn_rows,
+                       uint32_t* status, cudaStream_t stream);
+// dz[c, :] (bf16, pitch v^8, `bwd.cap` rows allocated) for the backward's compact rows from the kept logits;
+// fwd_pos maps a batch row to its row in `saved` (null: identity).
+int dz_from_saved(const void* saved, long long saved_rows, int v, const int* fwd_pos, const CompactBuffers& bwd,
+                  float inv_t, void* dz, cudaStream_t stream);
+int lmhead_bwd_from_dz_tc(const void* hidden, const void* w, const void* dz, long long n, int h, int v,
+                          void* grad_hidden, float* grad_w, int accumulate, const int* dyn_rows, uint32_t* status,
+                          cudaStream_t stream);
+
 // Launches a one-warp kernel whose bounded wait must expire after timeout_ms and set the status bit.
 int selftest_wait_timeout(uint32_t* status, unsigned timeout_ms, cudaStream_t stream);
 

@@ -163,6 +163,7 @@ struct SlabStore;  // output staging for TMA stores, defined below
 template <bool ENT>
 struct FwdEpilogue {
   static constexpr int kKernelId = kKTcFwd;
+  static constexpr bool kTwoPass = false;
   struct Params {
     const int32_t* targets;
     long long n;
@@ -273,6 +274,7 @@ struct SlabStore {
 
 struct DzEpilogue {
   static constexpr int kKernelId = kKTcDz;
+  static constexpr bool kTwoPass = false;
   struct Params {
     const int32_t* targets;   // indexed by global token row
     const float* lse;
@@ -329,8 +331,106 @@ struct DzEpilogue {
   __device__ __forceinline__ void end(const Params&, long long, int) {}
 };
 
+__device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
+  __half2 p = __floats2half2_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&p);
+}
+
+// Forward that also keeps the logits for the backward, so that the backward need not recompute
+// them: u[row, v] = z[row, v] * log2(e) / T - ref[row, tile] in fp16, where ref is the row's
+// running maximum once the 256-column tile has been seen (so u <= 0 and the entries that matter
+// for the softmax are the accurately stored ones), and ref[row, tile] in fp32.  The tile is swept
+// twice in TMEM: first for its row maxima, then for the exponentials and the stores.
+struct FwdSaveEpilogue {
+  static constexpr int kKernelId = kKTcFwdSave;
+  static constexpr bool kTwoPass = true;
+  struct Params {
+    const int32_t* targets;
+    long long n;
+    int v;
+    int vpad;      // row pitch of u
+    int n_tiles;   // row pitch of ref
+    float scale_log2;
+    float inv_t;
+    SoftmaxPartial* part;
+    float* zy;
+    __half* u;     // [n, vpad]
+    float* ref;    // [n, n_tiles]
+  };
+  static int make_c_map(const Params& p, CUtensorMap* map) {
+    return make_out_map(map, p.u, 2, p.v, p.n, p.vpad);  // 2-byte elements: a plain copy, the type does not matter
+  }
+  float m, s, tmax;
+  int y;
+  long long row;
+  uint8_t* cur;
+  __device__ __forceinline__ void begin(const Params& p, long long row_) {
+    row = row_;
+    m = -INFINITY; s = 0.f;
+    y = -1;
+    if (row < p.n) y = min(max(p.targets[row], 0), p.v - 1);
+  }
+  __device__ __forceinline__ void tile_begin() { tmax = -INFINITY; }
+  __device__ __forceinline__ void prepass(const Params& p, int col0, uint32_t (&r)[kEpiChunk]) {
+    if (col0 + kEpiChunk > p.v) {
+#pragma unroll
+      for (int j = 0; j < kEpiChunk; ++j)
+        if (col0 + j >= p.v) r[j] = 0xff800000u;  // -inf: columns past V do not exist
+    }
+#pragma unroll
+    for (int j = 0; j < kEpiChunk; ++j) tmax = fmaxf(tmax, bits_to_float(r[j]));
+  }
+  __device__ __forceinline__ void tile_ready(const Params& p, int tile) {
+    const float xm = tmax * p.scale_log2;
+    if (xm > m) {
+      s *= fast_exp2(m - xm);
+      m = xm;
+    }
+    if (row < p.n) p.ref[row * p.n_tiles + tile] = m;
+  }
+  __device__ __forceinline__ void chunk(const Params& p, int tile_row0, int col0, uint32_t (&r)[kEpiChunk],
+                                        SlabStore& st) {
+    if (col0 + kEpiChunk > p.v) {
+#pragma unroll
+      for (int j = 0; j < kEpiChunk; ++j)
+        if (col0 + j >= p.v) r[j] = 0xff800000u;
+    }
+    float x[kEpiChunk];
+    float acc = 0.f;
+#pragma unroll
+    for (int j = 0; j < kEpiChunk; ++j) {
+      x[j] = fmaf(bits_to_float(r[j]), p.scale_log2, -m);
+      acc += fast_exp2(x[j]);
+    }
+    s += acc;
+    if (y >= col0 && y < col0 + kEpiChunk) {
+      float zyv = 0.f;
+#pragma unroll
+      for (int j = 0; j < kEpiChunk; ++j)
+        if (col0 + j == y) zyv = bits_to_float(r[j]);
+      p.zy[row] = zyv * p.inv_t;
+    }
+    const int half = (col0 >> 5) & 1;
+    if (half == 0) cur = st.acquire();
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      uint4 w;
+      w.x = pack_half2(x[q * 8 + 0], x[q * 8 + 1]);
+      w.y = pack_half2(x[q * 8 + 2], x[q * 8 + 3]);
+      w.z = pack_half2(x[q * 8 + 4], x[q * 8 + 5]);
+      w.w = pack_half2(x[q * 8 + 6], x[q * 8 + 7]);
+      *st.piece(cur, half * 4 + q) = w;
+    }
+    if (half == 1) st.submit(cur, col0 - 32, tile_row0, col0 - 32 < p.v, false);
+  }
+  __device__ __forceinline__ void end(const Params& p, long long row_, int split) {
+    if (row_ < p.n) p.part[static_cast<long long>(split) * p.n + row_] = SoftmaxPartial{m * kLn2, s};
+  }
+};
+
 struct StoreBf16Epilogue {
   static constexpr int kKernelId = kKTcGradHidden;
+  static constexpr bool kTwoPass = false;
   struct Params {
     __nv_bfloat16* c;
     long long ldc;
@@ -362,6 +462,7 @@ struct StoreBf16Epilogue {
 
 struct StoreF32Epilogue {
   static constexpr int kKernelId = kKTcGradW;
+  static constexpr bool kTwoPass = false;
   struct Params {
     float* c;
     long long ldc;
@@ -562,6 +663,18 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           tcgen05_fence_after_sync();
         }
         const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(acc * BN);
+        if constexpr (Epi::kTwoPass) {
+          // first sweep over the accumulator tile: the epilogue learns the tile's row maxima
+          epi.tile_begin();
+#pragma unroll 1
+          for (int c = 0; c < BN / kEpiChunk; ++c) {
+            uint32_t r[kEpiChunk];
+            tmem_ld_32x32(taddr + static_cast<uint32_t>(c * kEpiChunk), r);
+            tmem_ld_wait();
+            epi.prepass(ep, nt * BN + c * kEpiChunk, r);
+          }
+          epi.tile_ready(ep, nt);
+        }
 #pragma unroll 1
         for (int c = 0; c < BN / kEpiChunk; ++c) {
           uint32_t r[kEpiChunk];
@@ -736,6 +849,28 @@ int lmhead_fwd_tc(const void* hidden, const void* w, const int32_t* targets, lon
   return launch_gemm<FwdEpilogue<false>, false, false>(a, b, splits, p, dyn, status, stream);
 }
 
+size_t lmhead_tc_saved_logits_bytes(long long n, int v) {
+  const size_t vpad = round_up(static_cast<size_t>(v), 8);
+  const size_t n_tiles = static_cast<size_t>((v + BN - 1) / BN);
+  return round_up(static_cast<size_t>(n) * vpad * 2, 256) + round_up(static_cast<size_t>(n) * n_tiles * 4, 256);
+}
+
+int lmhead_fwd_save_tc(const void* hidden, const void* w, const int32_t* targets, long long n, int h, int v,
+                       float inv_t, int splits, SoftmaxPartial* part, float* zy, void* saved, const int* dyn_rows,
+                       uint32_t* status, cudaStream_t stream) {
+  const Operand a{hidden, n, h, h};
+  const Operand b{w, v, h, h};
+  DynRows dyn;
+  dyn.rows = dyn_rows;
+  dyn.cap = n;
+  const int vpad = static_cast<int>(round_up(static_cast<size_t>(v), 8));
+  const int n_tiles = (v + BN - 1) / BN;
+  __half* u = static_cast<__half*>(saved);
+  float* ref = reinterpret_cast<float*>(static_cast<char*>(saved) + round_up(static_cast<size_t>(n) * vpad * 2, 256));
+  FwdSaveEpilogue::Params p{targets, n, v, vpad, n_tiles, inv_t * kLog2e, inv_t, part, zy, u, ref};
+  return launch_gemm<FwdSaveEpilogue, false, false>(a, b, splits, p, dyn, status, stream);
+}
+
 size_t lmhead_tc_bwd_ws_bytes(long long chunk_rows, long long /*n*/, int /*h*/, int v) {
   return bwd_ws_layout(chunk_rows, v);
 }
@@ -776,6 +911,29 @@ int lmhead_bwd_tc(const void* hidden_, const void* w_, const int32_t* targets, c
                                                               wp, dyn_k, status, stream)));
   }
   return A3PO_OK;
+}
+
+// The two contractions of the backward on a dz matrix that already exists for all n rows
+// (built from saved logits): grad_hidden = dz W, grad_w (+)= dz^T hidden.
+int lmhead_bwd_from_dz_tc(const void* hidden_, const void* w_, const void* dz_, long long n, int h, int v,
+                          void* grad_hidden_, float* grad_w, int accumulate, const int* dyn_rows, uint32_t* status,
+                          cudaStream_t stream) {
+  const __nv_bfloat16* hidden = static_cast<const __nv_bfloat16*>(hidden_);
+  const __nv_bfloat16* w = static_cast<const __nv_bfloat16*>(w_);
+  const __nv_bfloat16* dz = static_cast<const __nv_bfloat16*>(dz_);
+  const int vpad = static_cast<int>(round_up(static_cast<size_t>(v), 8));
+  DynRows dyn_m;
+  dyn_m.rows = dyn_rows;
+  dyn_m.cap = n;
+  DynRows dyn_k = dyn_m;
+  dyn_k.is_k = 1;
+  dyn_k.zero_when_empty = accumulate ? 0 : 1;
+  StoreBf16Epilogue::Params hp{static_cast<__nv_bfloat16*>(grad_hidden_), h, n, h};
+  A3PO_RETURN_IF((launch_gemm<StoreBf16Epilogue, false, true>(Operand{dz, n, v, vpad}, Operand{w, h, v, h}, 0, hp,
+                                                              dyn_m, status, stream)));
+  StoreF32Epilogue::Params wp{grad_w, h, v, h, accumulate ? 1 : 0};
+  return launch_gemm<StoreF32Epilogue, true, true>(Operand{dz, v, n, vpad}, Operand{hidden, h, n, h}, 0, wp, dyn_k,
+                                                   status, stream);
 }
 
 }  // namespace a3po

@@ -65,3 +65,49 @@ def test_chained_step_matches_oracle(name, kw):
     assert stats["n_clipped"] == ref["stats"]["n_clipped"]
     assert rel_fro(to_np64(gh), ref["gh"]) <= GRAD_FRO_RTOL * (1 if wl.dtype == "f32" else 3)
     assert rel_fro(to_np64(gw), ref["gw"]) <= GRAD_FRO_RTOL * (1 if wl.dtype == "f32" else 3)
+
+
+def _device_step(wl, behav, ws_bytes):
+    dt = a3po.A3PO_BF16
+    to_dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(DEV)
+    n = wl.N
+    out = dict(logp=torch.full((n,), 7.0, device=DEV), lse=torch.full((n,), 7.0, device=DEV),
+               grad_logp=torch.full((n,), 7.0, device=DEV), loss=torch.zeros(1, device=DEV),
+               grad_hidden=torch.full_like(wl.hidden, 7.0),
+               grad_w=torch.full((wl.V, wl.H), 7.0, dtype=torch.float32, device=DEV), stats=a3po.new_stats())
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    ws = a3po.new_workspace(ws_bytes)
+    a3po.a3po_train_step(wl.hidden, wl.w, to_dev(wl.targets), to_dev(behav), to_dev(wl.versions), wl.current_version,
+                         to_dev(wl.adv), to_dev(wl.mask), wl.clip_eps, out["logp"], out["lse"], out["grad_logp"],
+                         out["loss"], out["grad_hidden"], out["grad_w"], ws, stats=out["stats"], status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    return out
+
+
+@pytest.mark.parametrize("name,kw", [
+    ("1p5b", dict(V=8192 + 24, n_prompts=2, group=4, row_len=200, len_lo=30, len_hi=200)),
+    ("8b_packed", dict(V=2048 + 200, H=512, n_prompts=2, group=4, len_lo=20, len_hi=400)),
+])
+def test_kept_logits_step_matches_recomputing_step_and_oracle(name, kw):
+    """a3po_train_step with the recommended workspace (backward from kept fp16 logits) against the same call
+    with the minimum workspace (three calls, logits recomputed) and against the oracle."""
+    wl = workloads.make_workload(name, DEV, **kw)
+    ref = oracle_step(wl, wl.hidden, wl.w)          # also masks out tokens that sit on a clip bound
+    dt = a3po.A3PO_BF16
+    big = a3po.a3po_train_step_workspace_bytes(wl.N, wl.H, wl.V, dt)
+    small = a3po.a3po_train_step_min_workspace_bytes(wl.N, wl.H, wl.V, dt)
+    assert small < big
+    kept = _device_step(wl, ref["behav"], big)
+    recomputed = _device_step(wl, ref["behav"], small)
+    for out in (kept, recomputed):
+        assert np.max(np.abs(out["logp"].cpu().numpy() - ref["logp"])) <= 2e-3
+        assert abs(float(out["loss"].item()) - ref["loss"]) <= 5e-3 * max(ref["stats"]["abs_obj_mean"], 1e-12)
+        assert a3po.read_stats(out["stats"])["n_valid"] == ref["stats"]["n_valid"]
+        assert rel_fro(to_np64(out["grad_hidden"]), ref["gh"]) <= GRAD_FRO_RTOL * 3
+        assert rel_fro(to_np64(out["grad_w"]), ref["gw"]) <= GRAD_FRO_RTOL * 3
+        assert not to_np64(out["grad_hidden"])[wl.mask == 0].any()
+    # the two paths share the forward arithmetic up to the order of the online softmax
+    assert torch.allclose(kept["logp"], recomputed["logp"], atol=1e-4)
+    assert rel_fro(to_np64(kept["grad_w"]), to_np64(recomputed["grad_w"])) <= GRAD_FRO_RTOL
+    assert rel_fro(to_np64(kept["grad_hidden"]), to_np64(recomputed["grad_hidden"])) <= GRAD_FRO_RTOL
