@@ -360,7 +360,7 @@ struct FwdSaveEpilogue {
   static int make_c_map(const Params& p, CUtensorMap* map) {
     return make_out_map(map, p.u, 2, p.v, p.n, p.vpad);  // 2-byte elements: a plain copy, the type does not matter
   }
-  float m, s, tmax;
+  float m, s, tmax, ref_tile;
   int y;
   long long row;
   uint8_t* cur;
@@ -380,13 +380,16 @@ struct FwdSaveEpilogue {
 #pragma unroll
     for (int j = 0; j < kEpiChunk; ++j) tmax = fmaxf(tmax, bits_to_float(r[j]));
   }
+  // Fixes the tile's reference: the running maximum at this point (after the extra sweep for an
+  // item's first tile).  Later columns of the tile may exceed it, which only makes u slightly positive.
   __device__ __forceinline__ void tile_ready(const Params& p, int tile) {
-    const float xm = tmax * p.scale_log2;
+    const float xm = tmax * p.scale_log2;  // -inf unless the extra sweep ran
     if (xm > m) {
       s *= fast_exp2(m - xm);
       m = xm;
     }
-    if (row < p.n) p.ref[row * p.n_tiles + tile] = m;
+    ref_tile = m;
+    if (row < p.n) p.ref[row * p.n_tiles + tile] = ref_tile;
   }
   __device__ __forceinline__ void chunk(const Params& p, int tile_row0, int col0, uint32_t (&r)[kEpiChunk],
                                         SlabStore& st) {
@@ -395,12 +398,21 @@ struct FwdSaveEpilogue {
       for (int j = 0; j < kEpiChunk; ++j)
         if (col0 + j >= p.v) r[j] = 0xff800000u;
     }
+    float zmax = -INFINITY;
+#pragma unroll
+    for (int j = 0; j < kEpiChunk; ++j) zmax = fmaxf(zmax, bits_to_float(r[j]));
+    const float xm = zmax * p.scale_log2;
+    if (xm > m) {
+      s *= fast_exp2(m - xm);
+      m = xm;
+    }
+    const float back = ref_tile - m;  // <= 0: from the tile's reference to the running maximum
     float x[kEpiChunk];
     float acc = 0.f;
 #pragma unroll
     for (int j = 0; j < kEpiChunk; ++j) {
-      x[j] = fmaf(bits_to_float(r[j]), p.scale_log2, -m);
-      acc += fast_exp2(x[j]);
+      x[j] = fmaf(bits_to_float(r[j]), p.scale_log2, -ref_tile);
+      acc += fast_exp2(x[j] + back);
     }
     s += acc;
     if (y >= col0 && y < col0 + kEpiChunk) {
@@ -664,14 +676,17 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
         const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(acc * BN);
         if constexpr (Epi::kTwoPass) {
-          // first sweep over the accumulator tile: the epilogue learns the tile's row maxima
+          // an extra sweep over the first accumulator tile of an item: the epilogue learns the row maxima it
+          // uses as the first reference (later tiles take the running maximum they start with)
           epi.tile_begin();
+          if (nt == it.n_begin) {
 #pragma unroll 1
-          for (int c = 0; c < BN / kEpiChunk; ++c) {
-            uint32_t r[kEpiChunk];
-            tmem_ld_32x32(taddr + static_cast<uint32_t>(c * kEpiChunk), r);
-            tmem_ld_wait();
-            epi.prepass(ep, nt * BN + c * kEpiChunk, r);
+            for (int c = 0; c < BN / kEpiChunk; ++c) {
+              uint32_t r[kEpiChunk];
+              tmem_ld_32x32(taddr + static_cast<uint32_t>(c * kEpiChunk), r);
+              tmem_ld_wait();
+              epi.prepass(ep, nt * BN + c * kEpiChunk, r);
+            }
           }
           epi.tile_ready(ep, nt);
         }

@@ -16,9 +16,35 @@ namespace a3po {
 namespace {
 
 constexpr int kDzThreads = 256;
-constexpr int kColsPerThread = 8;
-constexpr int kSegCols = kDzThreads * kColsPerThread;  // 2048 columns per block iteration
-constexpr int kTileCols = 256;                          // column tile of the saving forward
+constexpr int kColsPerLoad = 8;                          // one 16-byte load of fp16
+constexpr int kLoadsPerThread = 2;                       // independent loads in flight per thread
+constexpr int kHalfSeg = kDzThreads * kColsPerLoad;      // 2048 columns
+constexpr int kSegCols = kHalfSeg * kLoadsPerThread;     // 4096 columns per block iteration
+constexpr int kTileCols = 256;                           // column tile of the saving forward
+
+__device__ __forceinline__ uint4 dz_piece(const uint4 raw, float shift, float g, int y, long long col0) {
+  const __half2* h2 = reinterpret_cast<const __half2*>(&raw);
+  float d[kColsPerLoad];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const float2 f = __half22float2(h2[j]);
+    d[2 * j] = -g * fast_exp2(f.x + shift);
+    d[2 * j + 1] = -g * fast_exp2(f.y + shift);
+  }
+  if (y >= col0 && y < col0 + kColsPerLoad) {
+#pragma unroll
+    for (int j = 0; j < kColsPerLoad; ++j)
+      if (col0 + j == y) d[j] += g;
+  }
+  __nv_bfloat162 b0 = __floats2bfloat162_rn(d[0], d[1]), b1 = __floats2bfloat162_rn(d[2], d[3]);
+  __nv_bfloat162 b2 = __floats2bfloat162_rn(d[4], d[5]), b3 = __floats2bfloat162_rn(d[6], d[7]);
+  uint4 out;
+  out.x = *reinterpret_cast<uint32_t*>(&b0);
+  out.y = *reinterpret_cast<uint32_t*>(&b1);
+  out.z = *reinterpret_cast<uint32_t*>(&b2);
+  out.w = *reinterpret_cast<uint32_t*>(&b3);
+  return out;
+}
 
 __global__ void __launch_bounds__(kDzThreads)
 dz_from_saved_kernel(const __half* __restrict__ u, const float* __restrict__ ref, long long vpad, int n_tiles, int v,
@@ -33,37 +59,26 @@ dz_from_saved_kernel(const __half* __restrict__ u, const float* __restrict__ ref
   for (long long item = blockIdx.x; item < items; item += gridDim.x) {
     const long long c = item / segs;
     const int seg = static_cast<int>(item % segs);
-    const long long col0 = static_cast<long long>(seg) * kSegCols + threadIdx.x * kColsPerThread;
-    if (col0 >= vpad) continue;
-    uint4 out = make_uint4(0u, 0u, 0u, 0u);
+    const long long col_a = static_cast<long long>(seg) * kSegCols + threadIdx.x * kColsPerLoad;
+    const long long col_b = col_a + kHalfSeg;
+    const bool in_a = col_a < vpad, in_b = col_b < vpad;
+    uint4 out_a = make_uint4(0u, 0u, 0u, 0u), out_b = out_a;
     const float g = (c < kept) ? g_c[c] * inv_t : 0.f;
     if (g != 0.f) {
       const long long orig = idx[c];                                  // row of the batch
       const long long src = fwd_pos ? fwd_pos[orig] : orig;           // its row in the forward's row space
-      const float shift = ref[src * n_tiles + col0 / kTileCols] - lse_c[c] * kLog2e;
+      const __half* urow = u + src * vpad;
+      uint4 raw_a = out_a, raw_b = out_a;
+      if (in_a) raw_a = __ldcs(reinterpret_cast<const uint4*>(urow + col_a));
+      if (in_b) raw_b = __ldcs(reinterpret_cast<const uint4*>(urow + col_b));
+      const float lse2 = lse_c[c] * kLog2e;
       const int y = min(max(targets_c[c], 0), v - 1);
-      const uint4 raw = __ldcs(reinterpret_cast<const uint4*>(u + src * vpad + col0));
-      const __half2* h2 = reinterpret_cast<const __half2*>(&raw);
-      float d[kColsPerThread];
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const float2 f = __half22float2(h2[j]);
-        d[2 * j] = -g * fast_exp2(f.x + shift);
-        d[2 * j + 1] = -g * fast_exp2(f.y + shift);
-      }
-      if (y >= col0 && y < col0 + kColsPerThread) {
-#pragma unroll
-        for (int j = 0; j < kColsPerThread; ++j)
-          if (col0 + j == y) d[j] += g;
-      }
-      __nv_bfloat162 b0 = __floats2bfloat162_rn(d[0], d[1]), b1 = __floats2bfloat162_rn(d[2], d[3]);
-      __nv_bfloat162 b2 = __floats2bfloat162_rn(d[4], d[5]), b3 = __floats2bfloat162_rn(d[6], d[7]);
-      out.x = *reinterpret_cast<uint32_t*>(&b0);
-      out.y = *reinterpret_cast<uint32_t*>(&b1);
-      out.z = *reinterpret_cast<uint32_t*>(&b2);
-      out.w = *reinterpret_cast<uint32_t*>(&b3);
+      const float* rrow = ref + src * n_tiles;
+      if (in_a) out_a = dz_piece(raw_a, rrow[col_a / kTileCols] - lse2, g, y, col_a);
+      if (in_b) out_b = dz_piece(raw_b, rrow[col_b / kTileCols] - lse2, g, y, col_b);
     }
-    __stcs(reinterpret_cast<uint4*>(dz + c * vpad + col0), out);
+    if (in_a) __stcs(reinterpret_cast<uint4*>(dz + c * vpad + col_a), out_a);
+    if (in_b) __stcs(reinterpret_cast<uint4*>(dz + c * vpad + col_b), out_b);
   }
 }
 
