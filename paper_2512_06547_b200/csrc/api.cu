@@ -426,8 +426,11 @@ size_t a3po_train_step_workspace_bytes(int64_t N, int H, int V, a3po_dtype dt) {
   if (b > a) a = b;
   if (c > a) a = c;
   if (dt == A3PO_BF16 && N > 0) {
+    // Keeping the logits costs N x V x 4 bytes of workspace (kept logits + dz, both for all N rows since the
+    // number of rows that take part is only known on the device).  It is recommended up to 96 GiB; beyond that
+    // the recommendation is the recomputing path's size (a caller may still pass more).
     const size_t d = saved_step_layout(N, H, V).total;
-    if (d > a) a = d;
+    if (d > a && d <= (static_cast<size_t>(96) << 30)) a = d;
   }
   return a;
 }

@@ -29,7 +29,10 @@ def _run_fullsize(name, n_sample_rows, seed):
     n, h, v = wl.N, wl.H, wl.V
     rng = np.random.default_rng(seed)
     targets, mask = _to_dev(wl.targets), _to_dev(wl.mask)
-    ws = a3po.new_workspace(a3po.a3po_train_step_workspace_bytes(n, h, v, a3po.A3PO_BF16))
+    dt = a3po.A3PO_BF16
+    ws = a3po.new_workspace(max(a3po.a3po_token_logprobs_workspace_bytes(n, h, v, dt, 0),
+                                a3po.a3po_token_logprobs_workspace_bytes(n, h, v, dt, 1),
+                                a3po.a3po_loss_workspace_bytes(n)))
     logp, lse = torch.empty(n, device=DEV), torch.empty(n, device=DEV)
     status = torch.zeros(1, dtype=torch.int32, device=DEV)
 
@@ -106,3 +109,50 @@ def test_8b_full_size():
 def test_8b_packed_full_size():
     """Packed varlen batch, ~1.1 M tokens, H=4096, per-token mask drops, ragged last row tile."""
     _run_fullsize("8b_packed", 48, seed=3)
+
+
+def test_1p5b_full_size_train_step():
+    """a3po_train_step (the call bench.py times; backward from kept logits) on the full 1.5B-shaped batch:
+    sampled rows of logp, grad_logp and grad_hidden against the oracle's own chain, grad_w by its property."""
+    wl = workloads.make_workload("1p5b", DEV)
+    n, h, v = wl.N, wl.H, wl.V
+    rng = np.random.default_rng(11)
+    valid_rows = np.flatnonzero(wl.mask)
+    idx = np.unique(np.concatenate([valid_rows[[0, -1]], rng.choice(valid_rows, 94, replace=False)]))
+    idx_t = torch.from_numpy(idx).to(DEV)
+    hn, wn = to_np64(wl.hidden[idx_t]), to_np64(wl.w)
+    logp_ref, _ = orc.token_logprobs_fwd(hn, wn, wl.targets[idx])
+    # behaviour log-probs: the recipe (current + noise) where the oracle knows "current", a plausible stand-in elsewhere
+    behav = np.minimum(-(np.log(v) + 0.5) + rng.standard_normal(n), 0).astype(np.float32)
+    behav[idx] = workloads.behav_logp_from(logp_ref, wl.behav_noise[idx])
+    m_total = int(wl.mask.sum())
+
+    dt = a3po.A3PO_BF16
+    ws = a3po.new_workspace(a3po.a3po_train_step_workspace_bytes(n, h, v, dt))
+    logp, lse, grad_logp = (torch.empty(n, device=DEV) for _ in range(3))
+    loss = torch.zeros(1, device=DEV)
+    stats = a3po.new_stats()
+    grad_hidden = torch.empty_like(wl.hidden)
+    grad_w = torch.empty((v, h), dtype=torch.float32, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    a3po.a3po_train_step(wl.hidden, wl.w, _to_dev(wl.targets), _to_dev(behav), _to_dev(wl.versions),
+                         wl.current_version, _to_dev(wl.adv), _to_dev(wl.mask), wl.clip_eps, logp, lse, grad_logp, loss,
+                         grad_hidden, grad_w, ws, stats=stats, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0 and a3po.read_stats(stats)["n_valid"] == m_total
+
+    assert np.max(np.abs(logp.cpu().numpy()[idx] - logp_ref)) <= LOGP_TOL_BF16
+    sub = (logp_ref, behav[idx], wl.versions[idx], wl.current_version, wl.adv[idx], wl.mask[idx], wl.clip_eps)
+    terms = orc.loss_terms(*sub)
+    g_ref = orc.loss_bwd(*sub, grad_loss=len(idx) / m_total)          # the mean runs over all M valid tokens
+    safe = terms["margin"] > 1e-2 * terms["r"]                         # away from the clip bounds (bf16 logp error)
+    assert safe.sum() >= 60
+    g_gpu = grad_logp.cpu().numpy()[idx]
+    assert np.max(np.abs(g_gpu[safe] - g_ref[safe])) <= 1e-2 * np.max(np.abs(g_ref)) + 1e-12
+    gh_ref, _ = orc.token_logprobs_bwd(hn[safe], wn, wl.targets[idx][safe], g_ref[safe])
+    assert rel_fro(to_np64(grad_hidden[idx_t[torch.from_numpy(safe)]]), gh_ref) <= 3 * GRAD_FRO_RTOL
+    assert not grad_hidden[_to_dev(np.flatnonzero(wl.mask == 0)[:2048])].float().abs().sum().item()
+    col_sum = grad_w.sum(dim=0, dtype=torch.float64)
+    col_abs = grad_w.abs().sum(dim=0, dtype=torch.float64)
+    assert float((col_sum.abs() / col_abs.clamp_min(1e-30)).max()) <= 2e-2
+    assert torch.isfinite(grad_w).all() and torch.isfinite(loss).all()
