@@ -32,6 +32,20 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 METRIC = "logprob+A-3PO loss fwd/bwd tokens/s; % of bf16 TC peak & HBM roofline"
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under profiles/.
+# GEMM kernels (profiles/gemm_tn_small_case_ncu_full.md): bytes per row that takes part, taken on the --small case
+# (2244 rows, H=1536, V=151936) and scaled by the rows of the launch (W re-reads and the kept logits / dz both grow
+# with the rows).  Only valid for that H and V; reset an entry to None when its kernel changes.
+NCU_TRAFFIC_PER_ROW_1P5B = {
+    "gemm_tn<fwd_logsoftmax+keep_logits>": (880.164e6 + 682.214e6) / 2244,
+    "gemm_tn<grad_hidden>": (1167.594e6 + 3.738e6) / 2244,
+    "gemm_tn<fwd_logsoftmax>": (879.835e6 + 3.917e6) / 2244,
+    "gemm_tn<dz>": (940.724e6 + 685.156e6) / 2244,
+    "gemm_tn<grad_w>": None,     # its traffic (874 MB of fp32 output + operands) does not scale with the rows
+}
+# Loss kernels (profiles/loss_kernels_16Mi_tokens_ncu_full.md): bytes per token at N = 2^24.
+NCU_TRAFFIC_PER_TOKEN_LOSS = {"loss_fwd_bwd": (285.231616e6 + 40.569600e6) / 16777216}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -232,7 +246,9 @@ def run_ours(args):
 
     # every rank draws its own shard of sequences (same shapes): weak scaling, no data-path collective
     seed = rank_seed(args.workload, rank)
-    shrink = dict(n_prompts=1, group=4) if args.small else {}   # --small: 4 sequences, for profiler captures
+    # --small: 4 sequences, for profiler captures; with a single group of 4 the Bernoulli rewards can all be
+    # equal (zero advantages, nothing to back-propagate), so its advantages are drawn N(0,1) per sequence instead
+    shrink = dict(n_prompts=1, group=4, reward_p=None) if args.small else {}
     wl = workloads.make_workload(args.workload, dev, seed=seed, **shrink)
     n, h, v = wl.N, wl.H, wl.V
     dt = a3po.A3PO_BF16 if wl.dtype == "bf16" else a3po.A3PO_F32
@@ -368,7 +384,10 @@ def run_ours(args):
     if dom["kernel"].startswith("gemm_tn"):
         achieved = dom["tflops"]
         roofline = {"bound": "tensor", "kernel": dom["kernel"], "achieved": achieved, "peak": sustained,
-                    "unit": "TFLOP/s", "frac": round(achieved / sustained, 4), "traffic": None,
+                    "unit": "TFLOP/s", "frac": round(achieved / sustained, 4),
+                    "traffic": (round(NCU_TRAFFIC_PER_ROW_1P5B[dom["kernel"]] * dom["rows"])
+                                if (h, v) == (1536, 151936) and NCU_TRAFFIC_PER_ROW_1P5B.get(dom["kernel"]) else None),
+                    "algorithmic_flops_per_launch": 2.0 * dom["rows"] * v * h,
                     "peak_source": f"{peaks['_source']} cuBLAS bf16, sustained (kernel timed inside a long step)",
                     "peak_burst": peaks["bf16_tflops"], "frac_of_burst": round(achieved / peaks["bf16_tflops"], 4),
                     "frac_of_nominal_2250": round(achieved / 2250.0, 4),
@@ -490,7 +509,9 @@ def run_loss_sweep(args):
                    "l2": "flushed between iterations" if flush is not None else "inputs exceed L2"},
         "roofline": {"bound": "hbm", "kernel": "loss_fwd_bwd", "achieved": round(best["kernel_gbs"], 1),
                      "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": round(best["kernel_gbs"] / peaks["hbm_gbs"], 4),
-                     "frac_of_nominal_8000": round(best["kernel_gbs"] / 8000.0, 4), "traffic": None,
+                     "frac_of_nominal_8000": round(best["kernel_gbs"] / 8000.0, 4),
+                     "traffic": round(NCU_TRAFFIC_PER_TOKEN_LOSS["loss_fwd_bwd"] * n),
+                     "algorithmic_bytes_per_launch": 21 * n,
                      "peak_source": f"{peaks['_source']} copy bandwidth"},
         "loss_kernels": results, "clocks": clocks, "gpu_launches": None, "e2e": None, "cpu_baseline": None,
     }
