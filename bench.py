@@ -166,7 +166,8 @@ def make_oracle_sample(name, rows):
     idx = np.flatnonzero(wl.mask)[:rows]
     hidden, w = workloads.lm_head_operands(len(idx), wl.H, wl.V, wl.dtype, wl.meta["seed"], "cpu")
     noise = wl.behav_noise[idx]
-    return dict(hidden=hidden.float().numpy(), w=w.float().numpy(), targets=wl.targets[idx],
+    # widened to float64 once, here: the oracle would otherwise widen W (V x H) again on every call
+    return dict(hidden=hidden.double().numpy(), w=w.double().numpy(), targets=wl.targets[idx],
                 versions=wl.versions[idx], current_version=wl.current_version, adv=wl.adv[idx],
                 mask=wl.mask[idx], clip_eps=wl.clip_eps, rows=len(idx),
                 behav_from=lambda logp: workloads.behav_logp_from(logp, noise))

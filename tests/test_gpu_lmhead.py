@@ -95,9 +95,12 @@ def test_fp32_shapes(n, h, v):
     _check_fwd_bwd(n, h, v, "f32", seed=100 + n, inv_t=0.9)
 
 
-@pytest.mark.parametrize("n,h,v", [(515, 1536, 4096 + 37), (131, 256, 777), (128, 64, 256), (300, 4096, 2048 + 8)])
+@pytest.mark.parametrize("n,h,v", [(515, 1536, 4096 + 37), (131, 256, 777), (128, 64, 256), (300, 4096, 2048 + 8),
+                                   (257, 72, 1000), (64, 8, 9), (1, 200, 300)])
 def test_bf16_shrunken_shapes(n, h, v):
-    """Same H as the 1.5B / 8B heads, shrunken V and N with ragged row and vocabulary tails."""
+    """Same H as the 1.5B / 8B heads, shrunken V and N with ragged row and vocabulary tails; also hidden sizes
+    that are not a multiple of the 64-wide K block (72, 8, 200: the K tail is zero-filled by the TMA loads), a
+    vocabulary smaller than one column tile and a single row."""
     _check_fwd_bwd(n, h, v, "bf16", seed=200 + n)
 
 
