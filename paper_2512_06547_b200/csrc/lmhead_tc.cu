@@ -4,6 +4,7 @@
 //     C[M, N] = A[M, K] * B[N, K]^T,
 // and differs only in its epilogue:
 //   forward      A = hidden, B = W           online (max, sum-exp) per row + target gather
+//   forward+keep same, and the shifted logits are kept in fp16 for a backward without recomputation
 //   dz           A = hidden, B = W           dz = g (1[v = y] - exp(z - lse)) -> bf16 chunk of rows
 //   grad_hidden  A = dz,     B = W^T         bf16 store            (W read in place as an N-major operand)
 //   grad_w       A = dz^T,   B = hidden^T    fp32 store/accumulate (both read in place, M-/N-major)
@@ -13,7 +14,9 @@
 // quarter each, one accumulator row per thread).  Operand tiles (128 x 64 and 256 x 64 bf16,
 // 128-byte swizzle) move through a 4-stage shared-memory ring guarded by full/empty mbarriers;
 // the 128 x 256 fp32 accumulator is double-buffered in TMEM (2 x 256 columns) so the epilogue
-// of tile i overlaps the MMAs of tile i+1.  Logits never leave TMEM/registers.
+// of tile i overlaps the MMAs of tile i+1.  Output tiles (kept logits, dz, gradients) leave through
+// two swizzled shared-memory slabs and TMA tile stores.  The full logits matrix never exists: the
+// plain forward keeps nothing, the keeping forward writes only the rows that take part, into scratch.
 //
 // Every mbarrier wait is bounded; on expiry the CTA raises A3PO_STATUS_WAIT_TIMEOUT in the
 // caller's status word, releases its TMEM and exits.
@@ -337,10 +340,11 @@ __device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
 }
 
 // Forward that also keeps the logits for the backward, so that the backward need not recompute
-// them: u[row, v] = z[row, v] * log2(e) / T - ref[row, tile] in fp16, where ref is the row's
-// running maximum once the 256-column tile has been seen (so u <= 0 and the entries that matter
-// for the softmax are the accurately stored ones), and ref[row, tile] in fp32.  The tile is swept
-// twice in TMEM: first for its row maxima, then for the exponentials and the stores.
+// them: u[row, v] = z[row, v] * log2(e) / T - ref[row, tile] in fp16 and ref[row, tile] in fp32,
+// where ref is the row's running maximum when the 256-column tile starts (u is then near or below
+// zero, so the entries that matter for the softmax are the accurately stored ones).  The first tile
+// of a work item has no running maximum yet: it is swept twice in TMEM, first for its row maxima,
+// then for the exponentials and the stores.
 struct FwdSaveEpilogue {
   static constexpr int kKernelId = kKTcFwdSave;
   static constexpr bool kTwoPass = true;
