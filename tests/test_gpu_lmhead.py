@@ -96,11 +96,12 @@ def test_fp32_shapes(n, h, v):
 
 
 @pytest.mark.parametrize("n,h,v", [(515, 1536, 4096 + 37), (131, 256, 777), (128, 64, 256), (300, 4096, 2048 + 8),
-                                   (257, 72, 1000), (64, 8, 9), (1, 200, 300)])
+                                   (257, 72, 1000), (64, 8, 9), (1, 200, 300), (33, 12, 50)])
 def test_bf16_shrunken_shapes(n, h, v):
     """Same H as the 1.5B / 8B heads, shrunken V and N with ragged row and vocabulary tails; also hidden sizes
     that are not a multiple of the 64-wide K block (72, 8, 200: the K tail is zero-filled by the TMA loads), a
-    vocabulary smaller than one column tile and a single row."""
+    vocabulary smaller than one column tile, a single row, and a hidden size (12) whose rows are not 16-byte
+    multiples, which the tensor-core path rejects and the FP32-pipe kernels take."""
     _check_fwd_bwd(n, h, v, "bf16", seed=200 + n)
 
 
