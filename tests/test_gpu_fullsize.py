@@ -156,3 +156,20 @@ def test_1p5b_full_size_train_step():
     col_abs = grad_w.abs().sum(dim=0, dtype=torch.float64)
     assert float((col_sum.abs() / col_abs.clamp_min(1e-30)).max()) <= 2e-2
     assert torch.isfinite(grad_w).all() and torch.isfinite(loss).all()
+
+
+def test_loss_only_16Mi_tokens():
+    """Loss-only sweep workload at 2^24 tokens (the size the bandwidth figures are quoted from, one below the
+    largest): loss, diagnostics and every token's gradient against the oracle, both value distributions."""
+    n = 1 << 24
+    for correlated in (False, True):
+        inp = workloads.loss_sweep(n, correlated=correlated)
+        dev = {k: _to_dev(inp[k]) for k in ("logp", "behav_logp", "versions", "adv", "mask")}
+        ws = a3po.new_workspace(a3po.a3po_loss_workspace_bytes(n))
+        loss = torch.zeros(1, device=DEV)
+        stats = a3po.new_stats()
+        grad = torch.empty(n, device=DEV)
+        a3po.a3po_loss_fwd_bwd(dev["logp"], dev["behav_logp"], dev["versions"], inp["current_version"], dev["adv"],
+                               dev["mask"], inp["clip_eps"], loss, grad, ws, stats=stats)
+        torch.cuda.synchronize()
+        check_loss_outputs(inp, float(loss.item()), a3po.read_stats(stats), grad.cpu().numpy())
