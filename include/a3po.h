@@ -115,6 +115,41 @@ int a3po_token_logprobs_bwd(const void* hidden, const void* w, const int32_t* ta
                             uint32_t* status, void* stream);
 
 /* --------------------------------------------------------------------------------------------
+ * Forward / backward pair that shares the logits instead of recomputing them (bf16 inputs only;
+ * no counterpart in the paper).  For callers whose forward and backward are separate calls, as
+ * under an autograd engine:
+ *
+ *   a3po_token_logprobs_fwd_keep  = a3po_token_logprobs_fwd (same logp, lse; rows with row_mask 0
+ *       are skipped) that also fills `kept` with the logits of the rows that took part: fp16,
+ *       shifted by a per-row reference per 256 vocabulary columns so that the entries that matter
+ *       for the softmax are stored accurately, plus the references and the row map.
+ *   a3po_token_logprobs_bwd_kept  = a3po_token_logprobs_bwd (same grad_hidden, grad_w within the
+ *       gradient tolerance) that turns `kept` into dz in one streaming pass and runs only the two
+ *       gradient contractions: 4 N V H flops instead of 6 N V H for the backward.
+ *
+ * `kept`: device buffer of a3po_kept_logits_bytes(N, V) bytes (about 2 N V bytes), 256-byte
+ * aligned, written by the forward, read by the backward; hidden, w, targets and lse must be the
+ * forward's.  Rows skipped by the forward must have grad_logp == 0.  Both calls return
+ * A3PO_ERR_UNSUPPORTED for shapes the tensor-core path does not take (H % 8 != 0): use the plain
+ * pair then.  ws: at least the matching *_workspace_bytes.
+ * ------------------------------------------------------------------------------------------ */
+size_t a3po_kept_logits_bytes(int64_t N, int V);
+size_t a3po_token_logprobs_fwd_keep_workspace_bytes(int64_t N, int H, int V);
+size_t a3po_token_logprobs_bwd_kept_workspace_bytes(int64_t N, int H, int V);
+
+int a3po_token_logprobs_fwd_keep(const void* hidden, const void* w, const int32_t* targets,
+                                 const uint8_t* row_mask, int64_t N, int H, int V,
+                                 float inv_temperature, float* logp, float* lse, void* kept,
+                                 size_t kept_bytes, void* ws, size_t ws_bytes, uint32_t* status,
+                                 void* stream);
+
+int a3po_token_logprobs_bwd_kept(const void* hidden, const void* w, const int32_t* targets,
+                                 const float* lse, const float* grad_logp, const void* kept,
+                                 size_t kept_bytes, int64_t N, int H, int V, float inv_temperature,
+                                 void* grad_hidden, float* grad_w, int accumulate_grad_w, void* ws,
+                                 size_t ws_bytes, uint32_t* status, void* stream);
+
+/* --------------------------------------------------------------------------------------------
  * A-3PO loss (Eq. 2 with the proximal policy of Eq. 3 and the coefficient of Eq. 4; argument
  * names follow Listing 1: behav_logp = old_logp, logp = logprobs, versions, current_version).
  *

@@ -62,6 +62,15 @@ _SIGNATURES = {
     "a3po_grpo_advantages": (c_int, [c_void_p, c_int, c_int, c_void_p, c_int64, c_float, c_void_p, c_void_p, c_size_t,
                                      c_void_p]),
     "a3po_selftest_wait_timeout": (c_int, [c_void_p, ctypes.c_uint, c_void_p]),
+    "a3po_kept_logits_bytes": (c_size_t, [c_int64, c_int]),
+    "a3po_token_logprobs_fwd_keep_workspace_bytes": (c_size_t, [c_int64, c_int, c_int]),
+    "a3po_token_logprobs_bwd_kept_workspace_bytes": (c_size_t, [c_int64, c_int, c_int]),
+    "a3po_token_logprobs_fwd_keep": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_int, c_int, c_float,
+                                             c_void_p, c_void_p, c_void_p, c_size_t, c_void_p, c_size_t, c_void_p,
+                                             c_void_p]),
+    "a3po_token_logprobs_bwd_kept": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t,
+                                             c_int64, c_int, c_int, c_float, c_void_p, c_void_p, c_int, c_void_p,
+                                             c_size_t, c_void_p, c_void_p]),
     "a3po_train_step_min_workspace_bytes": (c_size_t, [c_int64, c_int, c_int, c_int]),
     "a3po_train_step": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_int, c_int, c_int,
                                 c_int32, c_float, c_float, c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_void_p,
@@ -209,6 +218,54 @@ def a3po_token_logprobs_bwd(hidden, w, targets, lse, grad_logp, grad_hidden, gra
                                                 int(bool(accumulate_grad_w)), _ptr(ws), ws.numel(), _ptr(status),
                                                 _stream(stream))
     _check("a3po_token_logprobs_bwd", rc)
+
+
+def a3po_kept_logits_bytes(N, V) -> int:
+    return load_library().a3po_kept_logits_bytes(N, V)
+
+
+def a3po_token_logprobs_fwd_keep_workspace_bytes(N, H, V) -> int:
+    return load_library().a3po_token_logprobs_fwd_keep_workspace_bytes(N, H, V)
+
+
+def a3po_token_logprobs_bwd_kept_workspace_bytes(N, H, V) -> int:
+    return load_library().a3po_token_logprobs_bwd_kept_workspace_bytes(N, H, V)
+
+
+def a3po_token_logprobs_fwd_keep(hidden, w, targets, logp, lse, kept, ws, *, row_mask=None, inv_temperature=1.0,
+                                 status=None, stream=None):
+    """Forward that also fills `kept` (uint8 buffer of a3po_kept_logits_bytes) for a3po_token_logprobs_bwd_kept."""
+    _want(hidden, torch.bfloat16, "hidden"); _want(w, torch.bfloat16, "w")
+    _want(targets, torch.int32, "targets"); _want(row_mask, torch.uint8, "row_mask")
+    _want(logp, torch.float32, "logp"); _want(lse, torch.float32, "lse")
+    _want(kept, torch.uint8, "kept"); _want(ws, torch.uint8, "ws"); _want(status, torch.int32, "status")
+    n, h = hidden.shape
+    v = w.shape[0]
+    if w.shape[1] != h or targets.numel() != n or logp.numel() != n or lse.numel() != n:
+        raise ValueError("shape mismatch")
+    rc = load_library().a3po_token_logprobs_fwd_keep(_ptr(hidden), _ptr(w), _ptr(targets), _ptr(row_mask), n, h, v,
+                                                     float(inv_temperature), _ptr(logp), _ptr(lse), _ptr(kept),
+                                                     kept.numel(), _ptr(ws), ws.numel(), _ptr(status), _stream(stream))
+    _check("a3po_token_logprobs_fwd_keep", rc)
+
+
+def a3po_token_logprobs_bwd_kept(hidden, w, targets, lse, grad_logp, kept, grad_hidden, grad_w, ws, *,
+                                 accumulate_grad_w=False, inv_temperature=1.0, status=None, stream=None):
+    """Backward from the logits kept by a3po_token_logprobs_fwd_keep (no recomputation of the LM head)."""
+    _want(hidden, torch.bfloat16, "hidden"); _want(w, torch.bfloat16, "w")
+    _want(grad_hidden, torch.bfloat16, "grad_hidden"); _want(targets, torch.int32, "targets")
+    _want(lse, torch.float32, "lse"); _want(grad_logp, torch.float32, "grad_logp")
+    _want(grad_w, torch.float32, "grad_w"); _want(kept, torch.uint8, "kept"); _want(ws, torch.uint8, "ws")
+    _want(status, torch.int32, "status")
+    n, h = hidden.shape
+    v = w.shape[0]
+    if w.shape[1] != h or grad_hidden.shape != hidden.shape or grad_w.shape != w.shape or grad_logp.numel() != n:
+        raise ValueError("shape mismatch")
+    rc = load_library().a3po_token_logprobs_bwd_kept(_ptr(hidden), _ptr(w), _ptr(targets), _ptr(lse), _ptr(grad_logp),
+                                                     _ptr(kept), kept.numel(), n, h, v, float(inv_temperature),
+                                                     _ptr(grad_hidden), _ptr(grad_w), int(bool(accumulate_grad_w)),
+                                                     _ptr(ws), ws.numel(), _ptr(status), _stream(stream))
+    _check("a3po_token_logprobs_bwd_kept", rc)
 
 
 # ------------------------------------------------------------------------------ loss

@@ -385,23 +385,120 @@ size_t a3po_train_step_stage_bytes(int64_t N, int H, a3po_dtype dt) {
   return stage_layout(N, H, dt).total;
 }
 
+// ------------------------------------------------------------------------------------------------
+// Forward that keeps its logits / backward that uses them (no recomputation of the LM head).
+// ------------------------------------------------------------------------------------------------
+namespace {
+// `kept` buffer: pos[N] (row of the batch -> row of the kept logits, -1 for rows that took no part), then the
+// kept logits proper (fp16 u and fp32 references, see lmhead_tc_saved_logits_bytes).
+size_t kept_pos_bytes(long long n) { return round_up(sizeof(int) * static_cast<size_t>(n > 0 ? n : 0), 256); }
+}  // namespace
+
+size_t a3po_kept_logits_bytes(int64_t N, int V) {
+  if (N < 0 || V <= 0) return 0;
+  return kept_pos_bytes(N) + lmhead_tc_saved_logits_bytes(N, V) + 256;
+}
+
+size_t a3po_token_logprobs_fwd_keep_workspace_bytes(int64_t N, int H, int V) {
+  if (N < 0 || H <= 0 || V <= 0) return 0;
+  return compact_ws_bytes(N, H, false) + fwd_ws_for(N, lmhead_tc_fwd_splits(N, V)) + 256;
+}
+
+size_t a3po_token_logprobs_bwd_kept_workspace_bytes(int64_t N, int H, int V) {
+  if (N < 0 || H <= 0 || V <= 0) return 0;
+  return compact_ws_bytes(N, H, true) + lmhead_tc_bwd_ws_bytes(compact_capacity(N), N, H, V) + 256;
+}
+
+int a3po_token_logprobs_fwd_keep(const void* hidden, const void* w, const int32_t* targets, const uint8_t* row_mask,
+                                 int64_t N, int H, int V, float inv_temperature, float* logp, float* lse, void* kept,
+                                 size_t kept_bytes, void* ws, size_t ws_bytes, uint32_t* status, void* stream_) {
+  A3PO_RETURN_IF(check_lmhead_args(hidden, w, targets, N, H, V, A3PO_BF16, inv_temperature));
+  if (N > 0 && (!logp || !lse)) return A3PO_ERR_INVALID_ARG;
+  if (N == 0) return A3PO_OK;
+  if (!use_tc(A3PO_BF16, hidden, w, N, H, V)) return A3PO_ERR_UNSUPPORTED;
+  if (!kept || !aligned_to(kept, 256) || kept_bytes < a3po_kept_logits_bytes(N, V)) return A3PO_ERR_WORKSPACE;
+  if (!ws || !aligned_to(ws, 256) || ws_bytes < a3po_token_logprobs_fwd_keep_workspace_bytes(N, H, V))
+    return A3PO_ERR_WORKSPACE;
+  cudaStream_t stream = as_stream(stream_);
+  const int splits = lmhead_tc_fwd_splits(N, V);
+  CompactBuffers cb;
+  size_t used = 0;
+  if (!compact_carve(ws, ws_bytes, N, H, false, &cb, &used)) return A3PO_ERR_WORKSPACE;
+  Arena arena(static_cast<char*>(ws) + used, ws_bytes - used);
+  SoftmaxPartial* part = arena.take<SoftmaxPartial>(static_cast<size_t>(N) * splits);
+  float* zy = arena.take<float>(static_cast<size_t>(N));
+  if (!arena.ok()) return A3PO_ERR_WORKSPACE;
+  int* kept_pos = static_cast<int*>(kept);
+  void* saved = static_cast<char*>(kept) + kept_pos_bytes(N);
+
+  A3PO_RETURN_IF(compact_rows(hidden, H, targets, row_mask, nullptr, nullptr, N, cb, stream));
+  A3PO_RETURN_IF(lmhead_fwd_save_tc(cb.hidden_c, w, cb.targets_c, N, H, V, inv_temperature, splits, part, zy, saved,
+                                    cb.count, status, stream));
+  const unsigned blocks = static_cast<unsigned>((N + kMergeThreads - 1) / kMergeThreads);
+  A3PO_LAUNCH(kKMergePartials, stream, (merge_partials_kernel<<<blocks, kMergeThreads, 0, stream>>>(
+                                           part, nullptr, zy, targets, row_mask, cb.pos, N, V, splits, logp, lse,
+                                           nullptr, status)));
+  A3PO_RETURN_IF(after_launch());
+  // the row map outlives the workspace: the backward finds each row's kept logits through it
+  if (cudaMemcpyAsync(kept_pos, cb.pos, sizeof(int) * static_cast<size_t>(N), cudaMemcpyDeviceToDevice, stream) !=
+      cudaSuccess) {
+    cudaGetLastError();
+    return A3PO_ERR_CUDA;
+  }
+  return A3PO_OK;
+}
+
+int a3po_token_logprobs_bwd_kept(const void* hidden, const void* w, const int32_t* targets, const float* lse,
+                                 const float* grad_logp, const void* kept, size_t kept_bytes, int64_t N, int H, int V,
+                                 float inv_temperature, void* grad_hidden, float* grad_w, int accumulate_grad_w,
+                                 void* ws, size_t ws_bytes, uint32_t* status, void* stream_) {
+  A3PO_RETURN_IF(check_lmhead_args(hidden, w, targets, N, H, V, A3PO_BF16, inv_temperature));
+  if (!grad_w || (N > 0 && (!lse || !grad_logp || !grad_hidden))) return A3PO_ERR_INVALID_ARG;
+  if (!aligned_to(grad_hidden, 16) || !aligned_to(grad_w, 16)) return A3PO_ERR_UNSUPPORTED;
+  if (N == 0) {
+    if (!accumulate_grad_w &&
+        cudaMemsetAsync(grad_w, 0, sizeof(float) * static_cast<size_t>(V) * H, as_stream(stream_)) != cudaSuccess) {
+      cudaGetLastError();
+      return A3PO_ERR_CUDA;
+    }
+    return A3PO_OK;
+  }
+  if (!use_tc(A3PO_BF16, hidden, w, N, H, V)) return A3PO_ERR_UNSUPPORTED;
+  if (!kept || !aligned_to(kept, 256) || kept_bytes < a3po_kept_logits_bytes(N, V)) return A3PO_ERR_WORKSPACE;
+  if (!ws || !aligned_to(ws, 256) || ws_bytes < a3po_token_logprobs_bwd_kept_workspace_bytes(N, H, V))
+    return A3PO_ERR_WORKSPACE;
+  cudaStream_t stream = as_stream(stream_);
+  CompactBuffers cb;
+  size_t used = 0;
+  if (!compact_carve(ws, ws_bytes, N, H, true, &cb, &used)) return A3PO_ERR_WORKSPACE;
+  void* dz = static_cast<char*>(ws) + used;
+  if (ws_bytes - used < lmhead_tc_bwd_ws_bytes(compact_capacity(N), N, H, V)) return A3PO_ERR_WORKSPACE;
+  const int* kept_pos = static_cast<const int*>(kept);
+  const void* saved = static_cast<const char*>(kept) + kept_pos_bytes(N);
+
+  // rows with a non-zero upstream gradient only; dz from the kept logits, then the two contractions
+  A3PO_RETURN_IF(compact_rows(hidden, H, targets, nullptr, grad_logp, lse, N, cb, stream));
+  A3PO_RETURN_IF(dz_from_saved(saved, N, V, kept_pos, cb, inv_temperature, dz, stream));
+  A3PO_RETURN_IF(lmhead_bwd_from_dz_tc(cb.hidden_c, w, dz, N, H, V, cb.grad_hidden_c, grad_w, accumulate_grad_w,
+                                       cb.count, status, stream));
+  return scatter_rows(cb.grad_hidden_c, H, cb.pos, N, grad_hidden, stream);
+}
+
 namespace {
 // Workspace of the step that keeps the forward's logits (fp16, shifted) for the backward.
 struct SavedStepLayout {
-  size_t fwd_compact, bwd_compact, partials, saved, dz, loss, total;
-  int splits;
+  size_t kept, kept_bytes, call_ws, call_ws_bytes, loss, total;
 };
 SavedStepLayout saved_step_layout(long long n, int h, int v) {
   SavedStepLayout s;
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = round_up(off + bytes, 256); return o; };
-  const long long cap = compact_capacity(n);
-  s.splits = lmhead_tc_fwd_splits(n, v);
-  s.fwd_compact = take(compact_ws_bytes(n, h, false));
-  s.bwd_compact = take(compact_ws_bytes(n, h, true));
-  s.partials = take(fwd_ws_for(n, s.splits));
-  s.saved = take(lmhead_tc_saved_logits_bytes(n, v));
-  s.dz = take(lmhead_tc_bwd_ws_bytes(cap, n, h, v));
+  s.kept_bytes = a3po_kept_logits_bytes(n, v);
+  s.kept = take(s.kept_bytes);
+  const size_t f = a3po_token_logprobs_fwd_keep_workspace_bytes(n, h, v);
+  const size_t b = a3po_token_logprobs_bwd_kept_workspace_bytes(n, h, v);
+  s.call_ws_bytes = f > b ? f : b;   // the forward's and the backward's scratch are never live together
+  s.call_ws = take(s.call_ws_bytes);
   s.loss = take(a3po_loss_workspace_bytes(n));
   s.total = off;
   return s;
@@ -445,8 +542,6 @@ int a3po_train_step(const void* hidden, const int32_t* targets, const float* beh
                                       !grad_logp)))
     return A3PO_ERR_INVALID_ARG;
   if (!ws || !aligned_to(ws, 256)) return A3PO_ERR_WORKSPACE;
-  cudaStream_t stream = as_stream(stream_);
-
   const bool keep_logits = N > 0 && use_tc(dt, hidden, w, N, H, V) && !env_flag("A3PO_NO_SAVED_LOGITS") &&
                            ws_bytes >= saved_step_layout(N, H, V).total && aligned_to(grad_hidden, 16) &&
                            aligned_to(grad_w, 16);
@@ -460,41 +555,17 @@ int a3po_train_step(const void* hidden, const int32_t* targets, const float* beh
                                    grad_w, accumulate_grad_w, ws, ws_bytes, status, stream_);
   }
 
-  // ---- forward on the rows with mask != 0, keeping shifted fp16 logits and their per-tile references
+  // ---- forward keeping its logits (rows with mask != 0), loss on every token, backward from the kept logits
   const SavedStepLayout lay = saved_step_layout(N, H, V);
   char* base = static_cast<char*>(ws);
-  CompactBuffers fwd_cb, bwd_cb;
-  size_t used = 0;
-  if (!compact_carve(base + lay.fwd_compact, compact_ws_bytes(N, H, false), N, H, false, &fwd_cb, &used) ||
-      !compact_carve(base + lay.bwd_compact, compact_ws_bytes(N, H, true), N, H, true, &bwd_cb, &used))
-    return A3PO_ERR_WORKSPACE;
-  Arena arena(base + lay.partials, fwd_ws_for(N, lay.splits));
-  SoftmaxPartial* part = arena.take<SoftmaxPartial>(static_cast<size_t>(N) * lay.splits);
-  arena.take<float>(static_cast<size_t>(N) * lay.splits);  // entropy partials: unused here, same layout
-  float* zy = arena.take<float>(static_cast<size_t>(N));
-  if (!arena.ok()) return A3PO_ERR_WORKSPACE;
-  void* saved = base + lay.saved;
-  void* dz = base + lay.dz;
-
-  A3PO_RETURN_IF(compact_rows(hidden, H, targets, mask, nullptr, nullptr, N, fwd_cb, stream));
-  A3PO_RETURN_IF(lmhead_fwd_save_tc(fwd_cb.hidden_c, w, fwd_cb.targets_c, N, H, V, inv_temperature, lay.splits, part,
-                                    zy, saved, fwd_cb.count, status, stream));
-  {
-    const unsigned blocks = static_cast<unsigned>((N + kMergeThreads - 1) / kMergeThreads);
-    A3PO_LAUNCH(kKMergePartials, stream, (merge_partials_kernel<<<blocks, kMergeThreads, 0, stream>>>(
-                                             part, nullptr, zy, targets, mask, fwd_cb.pos, N, V, lay.splits, logp,
-                                             lse, nullptr, status)));
-    A3PO_RETURN_IF(after_launch());
-  }
-  // ---- loss and dL/dlogp on every token
+  A3PO_RETURN_IF(a3po_token_logprobs_fwd_keep(hidden, w, targets, mask, N, H, V, inv_temperature, logp, lse,
+                                              base + lay.kept, lay.kept_bytes, base + lay.call_ws, lay.call_ws_bytes,
+                                              status, stream_));
   A3PO_RETURN_IF(a3po_loss_fwd_bwd(logp, behav_logp, versions, 0, nullptr, 0, current_version, adv, mask, N, clip_eps,
                                    1, loss, stats, grad_logp, base + lay.loss, a3po_loss_workspace_bytes(N), stream_));
-  // ---- backward on the rows with a non-zero upstream gradient: dz from the kept logits, two contractions
-  A3PO_RETURN_IF(compact_rows(hidden, H, targets, nullptr, grad_logp, lse, N, bwd_cb, stream));
-  A3PO_RETURN_IF(dz_from_saved(saved, N, V, fwd_cb.pos, bwd_cb, inv_temperature, dz, stream));
-  A3PO_RETURN_IF(lmhead_bwd_from_dz_tc(bwd_cb.hidden_c, w, dz, N, H, V, bwd_cb.grad_hidden_c, grad_w,
-                                       accumulate_grad_w, bwd_cb.count, status, stream));
-  return scatter_rows(bwd_cb.grad_hidden_c, H, bwd_cb.pos, N, grad_hidden, stream);
+  return a3po_token_logprobs_bwd_kept(hidden, w, targets, lse, grad_logp, base + lay.kept, lay.kept_bytes, N, H, V,
+                                      inv_temperature, grad_hidden, grad_w, accumulate_grad_w, base + lay.call_ws,
+                                      lay.call_ws_bytes, status, stream_);
 }
 
 int a3po_train_step_host(const void* h_hidden, const int32_t* h_targets, const float* h_behav_logp,

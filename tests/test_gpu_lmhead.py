@@ -183,3 +183,48 @@ def test_masked_and_zero_gradient_rows_are_skipped_consistently():
                                 accumulate=True)
             assert torch.equal(acc, base)                                              # accumulate: untouched
         assert not to_np64(gh)[g_np == 0].any()
+
+
+def test_forward_keep_backward_kept_pair_matches_oracle_and_plain_pair():
+    """The forward that keeps its logits and the backward that uses them, as two separate calls with the
+    upstream gradient computed in between (as under an autograd engine)."""
+    n, h, v = 700, 512, 5000 + 24
+    hidden, w, targets, g = _problem(n, h, v, "bf16", 91)
+    rng = np.random.default_rng(92)
+    mask_np = (rng.random(n) < 0.7).astype(np.uint8)
+    mask = torch.from_numpy(mask_np).to(DEV)
+    g = g * mask                                                # skipped rows carry no gradient
+    kept = a3po.new_workspace(a3po.a3po_kept_logits_bytes(n, v))
+    ws = a3po.new_workspace(max(a3po.a3po_token_logprobs_fwd_keep_workspace_bytes(n, h, v),
+                                a3po.a3po_token_logprobs_bwd_kept_workspace_bytes(n, h, v)))
+    logp, lse = torch.full((n,), 5.0, device=DEV), torch.full((n,), 5.0, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    a3po.a3po_token_logprobs_fwd_keep(hidden, w, targets, logp, lse, kept, ws, row_mask=mask, status=status)
+    ws.fill_(0xAB)                                              # the backward must not depend on the forward's scratch
+    gh = torch.full_like(hidden, 3.0)
+    gw = torch.full((v, h), 3.0, dtype=torch.float32, device=DEV)
+    a3po.a3po_token_logprobs_bwd_kept(hidden, w, targets, lse, g, kept, gh, gw, ws, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    hn, wn, tn = to_np64(hidden), to_np64(w), targets.cpu().numpy()
+    logp_ref, lse_ref = orc.token_logprobs_fwd(hn, wn, tn, row_mask=mask_np)
+    assert np.max(np.abs(logp.cpu().numpy() - logp_ref)) <= LOGP_TOL_BF16
+    assert np.max(np.abs(lse.cpu().numpy() - lse_ref)) <= LOGP_TOL_BF16
+    gh_ref, gw_ref = orc.token_logprobs_bwd(hn, wn, tn, to_np64(g))
+    assert rel_fro(to_np64(gh), gh_ref) <= GRAD_FRO_RTOL and rel_fro(to_np64(gw), gw_ref) <= GRAD_FRO_RTOL
+    assert not to_np64(gh)[to_np64(g) == 0].any()
+    # the plain pair gives the same gradients within the tolerance, and accumulation works on the kept pair too
+    gh2, gw2, _ = gpu_bwd(hidden, w, targets, lse, g)
+    assert rel_fro(to_np64(gw), to_np64(gw2)) <= GRAD_FRO_RTOL and rel_fro(to_np64(gh), to_np64(gh2)) <= GRAD_FRO_RTOL
+    base = torch.randn(v, h, device=DEV)
+    acc = base.clone()
+    a3po.a3po_token_logprobs_bwd_kept(hidden, w, targets, lse, g, kept, gh, acc, ws, accumulate_grad_w=True)
+    torch.cuda.synchronize()
+    assert rel_fro(to_np64(acc - base), gw_ref) <= GRAD_FRO_RTOL
+    # shapes outside the tensor-core path are refused, not silently computed another way
+    h_odd, w_odd, t_odd, g_odd = _problem(16, 12, 40, "bf16", 93)
+    with pytest.raises(a3po.A3poError) as e:
+        a3po.a3po_token_logprobs_fwd_keep(h_odd, w_odd, t_odd, torch.empty(16, device=DEV), torch.empty(16, device=DEV),
+                                          a3po.new_workspace(a3po.a3po_kept_logits_bytes(16, 40)),
+                                          a3po.new_workspace(a3po.a3po_token_logprobs_fwd_keep_workspace_bytes(16, 12, 40)))
+    assert e.value.code == -2
