@@ -242,7 +242,7 @@ def run_ours(args):
 
     def barrier():
         if world > 1:
-            dist.barrier()
+            dist.barrier(device_ids=[local_rank])
         torch.cuda.synchronize()
 
     # every rank draws its own shard of sequences (same shapes): weak scaling, no data-path collective

@@ -78,7 +78,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
   return true;
 }
 
-// ---------------------------------------------------------------- TMA (tiled, 2-D, no multicast)
+// ---------------------------------------------------------------- TMA (tiled, 2-D; every CTA fetches its own tiles)
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
 }
