@@ -1,26 +1,33 @@
 #!/usr/bin/env python
 """Benchmark of the A-3PO hot path: token log-probs fwd -> A-3PO loss fwd+bwd -> log-prob bwd.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload 1p5b|8b]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload 8b|1p5b|8b_packed]
 
-One "step" is one pass of the whole path over one synthetic batch shaped like the paper's
-1.5B set-up (H=1536, V=151,936, bf16, 16 sequences x 1024 rows).  Prints ONE JSON line.
+One "step" is one pass of the whole path (a3po_train_step) over one synthetic batch.  The default
+workload is the 8B-shaped batch of the paper's second set-up (H=4096, V=151,936, bf16, 64 sequences
+x 2048 rows), the largest padded configuration that fits one GPU.  Prints ONE JSON line.
 
-  value      whole-job valid (mask=1) tokens per second, inputs resident in HBM
+  value      whole-job valid (mask=1) tokens per second, inputs resident in HBM, per-kernel events off
   e2e        same metric through a3po_train_step_host: per-step inputs start in pinned host memory
   roofline   the dominant kernel's achieved TFLOP/s (algorithmic flops / CUDA-event duration of each
-             launch, recorded by the library on its launch stream) against the measured bf16 peak
+             launch, recorded by the library on its launch stream in a second, separately timed loop)
+             against the measured bf16 peak
+  configs    compact entries for the other named configurations: the 1.5B-shaped batch, the packed
+             long-response 8B batch and the loss-only sweep at 2^24 and 2^26 tokens, each timed in
+             its own window with its own clock samples
   cpu_baseline  the fp64 oracle timed on this machine's host cores on a bounded row sample
 
 --impl reference times the oracle alone (the paper ships no runnable reference implementation).
-With N > 1 (torchrun) every rank runs its own shard of sequences (weak scaling, no data-path
-collective); timing is bracketed by barriers and the maximum over ranks is reported.
+With --gpus N > 1 the script starts one process per GPU itself (unless it already runs under
+torchrun); every rank runs its own shard of sequences (weak scaling, no data-path collective); timing
+is bracketed by barriers and the maximum over ranks is reported.
 """
 from __future__ import annotations
 
 import argparse
 import json
 import os
+import socket
 import statistics
 import subprocess
 import sys
@@ -33,20 +40,17 @@ if ROOT not in sys.path:
 
 METRIC = "logprob+A-3PO loss fwd/bwd tokens/s; % of bf16 TC peak & HBM roofline"
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under profiles/.
-# GEMM kernels (profiles/gemm_tn_small_case_ncu_full.md): bytes per row that takes part, taken on the --small case
-# (2244 rows, H=1536, V=151936) and scaled by the rows of the launch (W re-reads and the kept logits / dz both grow
-# with the rows).  Only valid for that H and V; reset an entry to None when its kernel changes.
-NCU_TRAFFIC_PER_ROW_1P5B = {
-    "gemm_tn<fwd_logsoftmax+keep_logits>": (880.164e6 + 682.214e6) / 2244,
-    "gemm_tn<grad_hidden>": (1167.594e6 + 3.738e6) / 2244,
-    "gemm_tn<fwd_logsoftmax>": (879.835e6 + 3.917e6) / 2244,
-    "gemm_tn<dz>": (940.724e6 + 685.156e6) / 2244,
-    "gemm_tn<grad_w>": None,     # its traffic (874 MB of fp32 output + operands) does not scale with the rows
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant GEMM kernel, from the ncu captures
+# summarised under profiles/: bytes per row that takes part, taken on a --small case of the same H and V and
+# scaled by the rows of the launch (W re-reads and the kept matrix both grow with the rows).  An entry is
+# None until a capture of the current kernel exists for that shape.
+NCU_TRAFFIC_PER_ROW = {
+    # (H, V): {kernel name: bytes per row}
 }
 # Loss kernels (profiles/loss_kernels_16Mi_tokens_ncu_full.md): bytes per token at N = 2^24.
 NCU_TRAFFIC_PER_TOKEN_LOSS = {"loss_fwd_bwd": (285.231616e6 + 40.569600e6) / 16777216}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+LONG_REGION_S = 2.0      # a timed region longer than this runs under the power cap: the sustained peak applies
 
 
 def load_peaks():
@@ -62,24 +66,17 @@ def load_peaks():
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clocks and throttle reasons with nvidia-smi; windows are cut out by monotonic time."""
     QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    NAMES = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
 
     def __init__(self, gpu_index: int):
         self.gpu_index = gpu_index
         self.proc = None
         self.lines = []          # (arrival time, csv line)
         self.thread = None
-        self.t_begin = None
-        self.t_end = None
-
-    def mark_begin(self):
-        self.t_begin = time.monotonic()
-
-    def mark_end(self):
-        self.t_end = time.monotonic()
 
     def start(self):
         try:
@@ -97,19 +94,14 @@ class ClockSampler:
         for line in self.proc.stdout:
             self.lines.append((time.monotonic(), line.strip()))
 
-    def stop(self):
+    def window(self, t_begin, t_end):
+        """Summary of the samples that arrived in [t_begin + 50 ms, t_end]."""
         if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except subprocess.TimeoutExpired:
-            self.proc.kill()
+            return {"sm_mhz": None, "sm_max_mhz": None, "samples": 0, "reasons": ["nvidia-smi unavailable"]}
         sm, mx, power, reasons = [], [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        window = [ln for t, ln in self.lines
-                  if (self.t_begin is None or t >= self.t_begin + 0.05) and (self.t_end is None or t <= self.t_end)]
-        for ln in (window or [ln for _, ln in self.lines]):
+        for t, ln in list(self.lines):
+            if t < t_begin + 0.05 or t > t_end:
+                continue
             f = [x.strip() for x in ln.split(",")]
             if len(f) < 9:
                 continue
@@ -117,20 +109,31 @@ class ClockSampler:
                 sm.append(float(f[1])); mx.append(float(f[2])); power.append(float(f[3]))
             except ValueError:
                 continue
-            for name, val in zip(names, f[5:9]):
+            for name, val in zip(self.NAMES, f[5:9]):
                 if val.lower().startswith("active"):
                     reasons.add(name)
         if not sm:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+            return {"sm_mhz": None, "sm_max_mhz": None, "samples": 0, "reasons": ["no samples"]}
         return {"sm_mhz": statistics.median(sm), "sm_min_mhz": min(sm), "sm_max_mhz": max(mx),
                 "power_w_max": max(power), "samples": len(sm), "reasons": sorted(reasons)}
+
+    def stop(self):
+        if self.proc is None:
+            return
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
 
 
 WORKLOAD_TEXT = {
     "1p5b": "1.5B-shaped: H=1536, V=151936, bf16 hidden/W, fp32 accumulate; 16 sequences (2 prompts x group 8) "
             "x 1024 rows, response lengths U[256,1024] right-padded and masked; staleness U{0..4}",
     "8b": "8B-shaped: H=4096, V=151936, bf16; 64 sequences (8 prompts x group 8) x 2048 rows, "
-          "response lengths U[512,2048]; staleness U{0..8}",
+          "response lengths U[512,2048] right-padded and masked; staleness U{0..8}",
+    "8b_packed": "8B-shaped long-response packed batch: H=4096, V=151936, bf16; 256 sequences (16 prompts x group 16) "
+                 "packed (cu_seqlens), lengths U[512,8192]; staleness min(Geom(0.4)-1, 16); 5% of tokens masked out",
 }
 
 
@@ -178,7 +181,7 @@ def run_reference(args):
     if rank != 0:
         return
     # size the row sample so that warm-up + K steps take about two minutes on this machine's cores
-    probe = make_oracle_sample(args.workload, 32)
+    probe = make_oracle_sample(args.workload, 16)
     per_row = oracle_sample_step(probe) / probe["rows"]
     total_steps = args.steps + args.warmup
     rows = int(max(8, min(args.oracle_rows, 120.0 / max(total_steps, 1) / per_row)))
@@ -223,41 +226,58 @@ def reduce_over_ranks(times_ms, counts, device):
     return t.tolist(), c.tolist()
 
 
-def run_ours(args):
+def tensor_roofline(kernels, steps, h, v, region_s, peaks):
+    """Roofline object of the dominant GEMM kernel.  The peak is the measured cuBLAS bf16 figure that matches the
+    timed region: the burst figure for a short region, the sustained one when the region is long enough for the
+    board to sit at its power cap."""
+    gemms = [k for k in kernels if k["kernel"].startswith("gemm_tn")]
+    if not gemms:
+        return {"bound": "tensor", "kernel": None, "achieved": None, "peak": None, "unit": "TFLOP/s", "frac": None,
+                "traffic": None}
+    dom = gemms[0]
+    sustained = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
+    burst = peaks["bf16_tflops"]
+    long_region = region_s > LONG_REGION_S
+    peak = sustained if long_region else burst
+    per_row = NCU_TRAFFIC_PER_ROW.get((h, v), {}).get(dom["kernel"])
+    launches_per_step = max(dom["launches"] // max(steps, 1), 1)
+    all_flops = sum(2.0 * k["rows"] * v * h * steps for k in gemms)
+    all_ms = sum(k["ms_total"] for k in gemms)
+    return {"bound": "tensor", "kernel": dom["kernel"], "achieved": dom["tflops"], "peak": peak,
+            "unit": "TFLOP/s", "frac": round(dom["tflops"] / peak, 4),
+            "traffic": round(per_row * dom["rows"] / launches_per_step) if per_row else None,
+            "algorithmic_flops_per_launch": 2.0 * dom["rows"] * v * h / launches_per_step,
+            "launches_per_step": launches_per_step,
+            "peak_source": "%s cuBLAS bf16, %s (timed region %.1f s)" % (
+                peaks["_source"], "sustained" if long_region else "burst", region_s),
+            "peak_burst": burst, "frac_of_burst": round(dom["tflops"] / burst, 4),
+            "peak_sustained": sustained, "frac_of_sustained": round(dom["tflops"] / sustained, 4),
+            "frac_of_nominal_2250": round(dom["tflops"] / 2250.0, 4),
+            "all_gemm_tn_tflops": round(all_flops / (all_ms * 1e-3) / 1e12, 1)}
+
+
+def time_step_workload(name, args, sampler, dev, rank, world, barrier, *, steps, warmup, with_e2e, small=False):
+    """Builds the workload on `dev`, times `steps` passes of a3po_train_step with the per-kernel events off,
+    then the same number again with them on (kernel table), then optionally the host-input entry."""
     import numpy as np
     import torch
-    import torch.distributed as dist
 
     import paper_2512_06547_b200 as a3po
     from paper_2512_06547_b200 import workloads
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    torch.cuda.set_device(local_rank)
-    dev = torch.device("cuda", local_rank)
-    if world > 1:
-        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        dist.init_process_group("nccl", device_id=dev)
-
-    def barrier():
-        if world > 1:
-            dist.barrier(device_ids=[local_rank])
-        torch.cuda.synchronize()
-
-    # every rank draws its own shard of sequences (same shapes): weak scaling, no data-path collective
-    seed = rank_seed(args.workload, rank)
+    seed = rank_seed(name, rank)
     # --small: 4 sequences, for profiler captures; with a single group of 4 the Bernoulli rewards can all be
     # equal (zero advantages, nothing to back-propagate), so its advantages are drawn N(0,1) per sequence instead
-    shrink = dict(n_prompts=1, group=4, reward_p=None) if args.small else {}
-    wl = workloads.make_workload(args.workload, dev, seed=seed, **shrink)
+    shrink = dict(n_prompts=1, group=4, reward_p=None) if small else {}
+    wl = workloads.make_workload(name, dev, seed=seed, **shrink)
     n, h, v = wl.N, wl.H, wl.V
     dt = a3po.A3PO_BF16 if wl.dtype == "bf16" else a3po.A3PO_F32
     to_dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(dev)
     targets, versions, adv, mask = (to_dev(x) for x in (wl.targets, wl.versions, wl.adv, wl.mask))
     n_valid = int(wl.mask.sum())
 
-    ws = a3po.new_workspace(a3po.a3po_train_step_workspace_bytes(n, h, v, dt), dev)
+    ws_bytes = a3po.a3po_train_step_workspace_bytes(n, h, v, dt)
+    ws = a3po.new_workspace(ws_bytes, dev)
     logp = torch.empty(n, device=dev)
     lse = torch.empty(n, device=dev)
     grad_logp = torch.empty(n, device=dev)
@@ -280,71 +300,166 @@ def run_ours(args):
                                    grad_logp, ws, stats=stats)
             a3po.a3po_token_logprobs_bwd(wl.hidden, wl.w, targets, lse, grad_logp, grad_hidden, grad_w, ws,
                                          status=status)
-        else:                       # one call; the backward reuses the logits the forward kept in the workspace
+        else:                       # one call; the backward reuses what the forward kept in the workspace
             a3po.a3po_train_step(wl.hidden, wl.w, targets, behav, versions, wl.current_version, adv, mask,
                                  wl.clip_eps, logp, lse, grad_logp, loss, grad_hidden, grad_w, ws, stats=stats,
                                  status=status)
 
-    sampler = ClockSampler(local_rank)
-    if rank == 0:
-        sampler.start()          # started early: nvidia-smi needs a moment before its first sample
-    for _ in range(args.warmup):
+    def timed_loop(fn, k):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        t0 = time.monotonic()
+        e0.record()
+        for _ in range(k):
+            fn()
+        e1.record()
+        barrier()
+        t1 = time.monotonic()
+        return e0.elapsed_time(e1), (t0, t1)
+
+    for _ in range(warmup):
         step()
     barrier()
 
-    # ---- timed region: device-resident inputs
-    a3po.a3po_profile_enable(True)
-    a3po.a3po_profile_read()
-    launches0 = a3po.a3po_kernel_launch_count()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    sampler.mark_begin()
-    e0.record()
-    for _ in range(args.steps):
-        step()
-    e1.record()
-    barrier()
-    sampler.mark_end()
-    launches = a3po.a3po_kernel_launch_count() - launches0
+    # ---- timed region: device-resident inputs, per-kernel events off
     a3po.a3po_profile_enable(False)
-    per_kernel = a3po.a3po_profile_read()
-    clocks = sampler.stop() if rank == 0 else None
-    ms_total = e0.elapsed_time(e1)
+    launches0 = a3po.a3po_kernel_launch_count()
+    ms_total, win = timed_loop(step, steps)
+    launches = a3po.a3po_kernel_launch_count() - launches0
     if int(status.item()) != 0:
         raise RuntimeError(f"device status word = {int(status.item())}")
+    clocks = sampler.window(*win) if sampler else None
+
+    # ---- the same loop again with one CUDA-event pair around every launch: the kernel table
+    a3po.a3po_profile_enable(True)
+    a3po.a3po_profile_read()
+    ms_profiled, _ = timed_loop(step, steps)
+    a3po.a3po_profile_enable(False)
+    per_kernel = a3po.a3po_profile_read()
+
+    out = dict(wl=wl, n=n, h=h, v=v, n_valid=n_valid, ms_total=ms_total, ms_profiled=ms_profiled, launches=launches,
+               clocks=clocks, per_kernel=per_kernel, ws_bytes=ws_bytes, loss=float(loss.item()),
+               bwd_rows=int((grad_logp != 0).sum().item()), e2e=None)
 
     # ---- e2e: host-resident per-step inputs through the C ABI's host entry
-    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
-    h_hidden = wl.hidden.cpu().pin_memory()
-    h_targets, h_behav, h_versions, h_adv, h_mask = (pin(x) for x in (wl.targets, behav_host, wl.versions, wl.adv,
-                                                                       wl.mask))
-    h_loss = torch.zeros(1).pin_memory()
-    h_stats = torch.zeros(24, dtype=torch.uint8).pin_memory()
-    stage = a3po.new_workspace(a3po.a3po_train_step_stage_bytes(n, h, dt), dev)
+    if with_e2e:
+        pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+        h_hidden = wl.hidden.cpu().pin_memory()
+        h_targets, h_behav, h_versions, h_adv, h_mask = (pin(x) for x in (wl.targets, behav_host, wl.versions, wl.adv,
+                                                                           wl.mask))
+        h_loss = torch.zeros(1).pin_memory()
+        h_stats = torch.zeros(24, dtype=torch.uint8).pin_memory()
+        stage = a3po.new_workspace(a3po.a3po_train_step_stage_bytes(n, h, dt), dev)
 
-    def host_step():
-        a3po.a3po_train_step_host(h_hidden, h_targets, h_behav, h_versions, h_adv, h_mask, wl.current_version,
-                                  wl.clip_eps, wl.w, grad_w, grad_hidden, stage, ws, h_loss, h_stats=h_stats,
-                                  d_status=status)
-        torch.cuda.current_stream().synchronize()   # the step's loss is read on the host
-        return float(h_loss.item())
+        def host_step():
+            a3po.a3po_train_step_host(h_hidden, h_targets, h_behav, h_versions, h_adv, h_mask, wl.current_version,
+                                      wl.clip_eps, wl.w, grad_w, grad_hidden, stage, ws, h_loss, h_stats=h_stats,
+                                      d_status=status)
+            torch.cuda.current_stream().synchronize()   # the step's loss is read on the host
+            return float(h_loss.item())
 
-    for _ in range(min(args.warmup, 3)):
-        host_step()
-    barrier()
-    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    f0.record()
-    for _ in range(args.steps):
-        host_step()
-    f1.record()
-    barrier()
-    e2e_ms_total = f0.elapsed_time(f1)
-    h2d = h_hidden.numel() * h_hidden.element_size() + n * (4 + 4 + 4 + 4 + 1)
-    d2h = 4 + 24
+        for _ in range(min(warmup, 3)):
+            host_step()
+        e2e_ms_total, _ = timed_loop(host_step, steps)
+        # where the difference to the device-resident loop goes: the host->device copies, timed on their own
+        a3po.a3po_profile_enable(True)
+        a3po.a3po_profile_read()
+        for _ in range(3):
+            host_step()
+        a3po.a3po_profile_enable(False)
+        h2d_ms = [ms for k, ms in a3po.a3po_profile_read() if k == "h2d_copies"]
+        out["e2e"] = dict(ms_total=e2e_ms_total,
+                          h2d=h_hidden.numel() * h_hidden.element_size() + n * (4 + 4 + 4 + 4 + 1), d2h=4 + 24,
+                          h2d_ms=statistics.mean(h2d_ms) if h2d_ms else None)
+        del h_hidden, stage
+    del ws, grad_w, grad_hidden, wl.hidden, wl.w
+    torch.cuda.empty_cache()
+    return out
+
+
+def kernel_table(per_kernel, steps, fwd_rows, bwd_rows, n, v, h):
+    agg = {}
+    for name, ms in per_kernel:
+        a = agg.setdefault(name, [0, 0.0])
+        a[0] += 1
+        a[1] += ms
+    total = sum(x[1] for x in agg.values()) or 1.0
+    # Algorithmic flops per launch = 2 * (rows that take part) * V * H: the forward processes the rows with
+    # mask != 0, the backward contractions the rows whose upstream gradient is non-zero (padding and clipped
+    # tokens contribute nothing, so they are not counted as work whether or not a kernel skips them).
+    rows_of = {"gemm_tn<fwd_logsoftmax>": fwd_rows, "gemm_tn<fwd_logsoftmax+keep>": fwd_rows,
+               "gemm_tn<dz>": bwd_rows, "gemm_tn<grad_hidden>": bwd_rows, "gemm_tn<grad_w>": bwd_rows}
+    kernels = []
+    for name, (cnt, ms) in sorted(agg.items(), key=lambda kv: -kv[1][1]):
+        entry = {"kernel": name, "launches": cnt, "ms_total": round(ms, 4), "share": round(ms / total, 4)}
+        if name.startswith("gemm_tn"):
+            entry["rows"] = rows_of.get(name, n)
+            # a step may split a contraction over several launches (row chunks): flops are per step
+            entry["tflops"] = round(2.0 * entry["rows"] * v * h * steps / (ms * 1e-3) / 1e12, 1)
+        kernels.append(entry)
+    recomputes = any(k["kernel"] == "gemm_tn<dz>" for k in kernels)
+    step_flops = 2.0 * v * h * (fwd_rows + (3 if recomputes else 2) * bwd_rows)
+    return kernels, step_flops
+
+
+def steps_for(seconds_per_step, min_seconds, lo, hi):
+    k = int(min_seconds / max(seconds_per_step, 1e-6)) + 1
+    return max(lo, min(hi, k))
+
+
+def secondary_step_config(name, args, sampler, dev, barrier, peaks):
+    """Compact entry for another named configuration: timed in its own window of >= 1.5 s."""
+    import torch
+    # one short probe to size the loop, then the timed run
+    probe = time_step_workload(name, args, None, dev, 0, 1, barrier, steps=1, warmup=1, with_e2e=False)
+    per_step = probe["ms_total"] * 1e-3
+    steps = steps_for(per_step, 1.5, 2, 200)
+    r = time_step_workload(name, args, sampler, dev, 0, 1, barrier, steps=steps, warmup=3 if per_step < 1 else 1,
+                           with_e2e=False)
+    kernels, step_flops = kernel_table(r["per_kernel"], steps, r["n_valid"], r["bwd_rows"], r["n"], r["v"], r["h"])
+    ms_per_step = r["ms_total"] / steps
+    roof = tensor_roofline(kernels, steps, r["h"], r["v"], r["ms_total"] * 1e-3, peaks)
+    torch.cuda.empty_cache()
+    return {"workload": WORKLOAD_TEXT[name], "rows": r["n"], "valid_tokens": r["n_valid"], "steps": steps,
+            "ms_per_step": round(ms_per_step, 4), "value": round(r["n_valid"] / (ms_per_step * 1e-3), 1),
+            "unit": "tokens/s", "executed_tflops": round(step_flops / (ms_per_step * 1e-3) / 1e12, 1),
+            "workspace_gib": round(r["ws_bytes"] / 2 ** 30, 2),
+            "recompute_free": not any(k["kernel"] == "gemm_tn<dz>" for k in kernels),
+            "roofline": {k: roof[k] for k in ("bound", "kernel", "achieved", "peak", "unit", "frac", "frac_of_burst",
+                                              "frac_of_sustained", "peak_source") if k in roof},
+            "kernels": [{k: e[k] for k in ("kernel", "ms_total", "share", "tflops") if k in e} for e in kernels[:4]],
+            "clocks": r["clocks"]}
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier(device_ids=[local_rank])
+        torch.cuda.synchronize()
+
+    peaks = load_peaks()
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    if sampler:
+        sampler.start()          # started early: nvidia-smi needs a moment before its first sample
+    r = time_step_workload(args.workload, args, sampler, dev, rank, world, barrier, steps=args.steps,
+                           warmup=args.warmup, with_e2e=True, small=args.small)
+    n, h, v, n_valid = r["n"], r["h"], r["v"], r["n_valid"]
 
     # ---- max over ranks
     (ms_total, e2e_ms_total), (total_valid, total_rows) = reduce_over_ranks(
-        [ms_total, e2e_ms_total], [float(n_valid), float(n)], dev)
+        [r["ms_total"], r["e2e"]["ms_total"]], [float(n_valid), float(n)], dev)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -353,51 +468,21 @@ def run_ours(args):
     ms_per_step = ms_total / args.steps
     value = total_valid * args.steps / (ms_total * 1e-3)
     e2e_value = total_valid * args.steps / (e2e_ms_total * 1e-3)
+    kernels, step_flops = kernel_table(r["per_kernel"], args.steps, n_valid, r["bwd_rows"], n, v, h)
+    roofline = tensor_roofline(kernels, args.steps, h, v, ms_total * 1e-3, peaks)
 
-    # ---- roofline of the dominant kernel, from the per-launch CUDA events of the timed region
-    peaks = load_peaks()
-    agg = {}
-    for name, ms in per_kernel:
-        a = agg.setdefault(name, [0, 0.0])
-        a[0] += 1
-        a[1] += ms
-    kernel_total = sum(x[1] for x in agg.values()) or 1.0
-    # Algorithmic flops per launch = 2 * (rows that take part) * V * H: the forward processes the rows with
-    # mask != 0, the three backward contractions the rows whose upstream gradient is non-zero (padding and
-    # clipped tokens are skipped by the library, so they are not counted as work).
-    fwd_rows = n_valid
-    bwd_rows = int((grad_logp != 0).sum().item())
-    rows_of = {"gemm_tn<fwd_logsoftmax>": fwd_rows, "gemm_tn<fwd_logsoftmax+keep_logits>": fwd_rows,
-               "gemm_tn<dz>": bwd_rows, "gemm_tn<grad_hidden>": bwd_rows, "gemm_tn<grad_w>": bwd_rows}
-    # contractions actually executed per step: forward + (dz recompute unless the logits were kept) + two gradients
-    recomputes = any(name == "gemm_tn<dz>" for name in agg)
-    step_flops = 2.0 * v * h * (fwd_rows + (3 if recomputes else 2) * bwd_rows)
-    kernels = []
-    for name, (cnt, ms) in sorted(agg.items(), key=lambda kv: -kv[1][1]):
-        entry = {"kernel": name, "launches": cnt, "ms_total": round(ms, 4), "share": round(ms / kernel_total, 4)}
-        if name.startswith("gemm_tn"):
-            entry["rows"] = rows_of.get(name, n)
-            # a step may split a contraction over several launches (row chunks): flops are per step
-            entry["tflops"] = round(2.0 * entry["rows"] * v * h * args.steps / (ms * 1e-3) / 1e12, 1)
-        kernels.append(entry)
-    dom = kernels[0]
-    sustained = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
-    if dom["kernel"].startswith("gemm_tn"):
-        achieved = dom["tflops"]
-        roofline = {"bound": "tensor", "kernel": dom["kernel"], "achieved": achieved, "peak": sustained,
-                    "unit": "TFLOP/s", "frac": round(achieved / sustained, 4),
-                    "traffic": (round(NCU_TRAFFIC_PER_ROW_1P5B[dom["kernel"]] * dom["rows"])
-                                if (h, v) == (1536, 151936) and NCU_TRAFFIC_PER_ROW_1P5B.get(dom["kernel"]) else None),
-                    "algorithmic_flops_per_launch": 2.0 * dom["rows"] * v * h,
-                    "peak_source": f"{peaks['_source']} cuBLAS bf16, sustained (kernel timed inside a long step)",
-                    "peak_burst": peaks["bf16_tflops"], "frac_of_burst": round(achieved / peaks["bf16_tflops"], 4),
-                    "frac_of_nominal_2250": round(achieved / 2250.0, 4),
-                    "all_gemm_tn_tflops": round(
-                        sum(2.0 * k["rows"] * v * h * args.steps for k in kernels if k["kernel"].startswith("gemm_tn")) /
-                        (sum(k["ms_total"] for k in kernels if k["kernel"].startswith("gemm_tn")) * 1e-3) / 1e12, 1)}
-    else:
-        roofline = {"bound": "hbm", "kernel": dom["kernel"], "achieved": None, "peak": peaks["hbm_gbs"],
-                    "unit": "GB/s", "frac": None, "traffic": None}
+    # ---- the other named configurations, each in its own window (one GPU only)
+    configs = None
+    if world == 1 and not args.no_configs and not args.small:
+        configs = {}
+        for name in ("1p5b", "8b", "8b_packed"):
+            if name != args.workload:
+                configs[name] = secondary_step_config(name, args, sampler, dev, barrier, peaks)
+        for tokens in (1 << 24, 1 << 26):
+            configs["loss_sweep_2^%d" % (tokens.bit_length() - 1)] = loss_sweep_entry(
+                tokens, sampler, dev, peaks, min_seconds=1.5)
+    if sampler:
+        sampler.stop()
 
     # ---- oracle beside it (rank 0, bounded sample)
     cpu_baseline = None
@@ -409,6 +494,7 @@ def run_ours(args):
                         "sample": f"the first {sample['rows']} valid rows of the batch at full H and V, one step, "
                                   "fp64 numpy"}
 
+    wl = r["wl"]
     line = {
         "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
@@ -416,19 +502,23 @@ def run_ours(args):
         "config": {"workload": WORKLOAD_TEXT[args.workload] + (" [--small: 4 sequences only]" if args.small else ""),
                    "rows_per_gpu": n, "valid_tokens_per_gpu": n_valid,
                    "H": h, "V": v, "parallelism": f"dp{world} (independent shards)",
-                   "l2": "no flush: W (%.0f MB) and the dz scratch are larger than the 126 MB L2"
+                   "workspace_gib": round(r["ws_bytes"] / 2 ** 30, 2),
+                   "l2": "no flush: W (%.0f MB) and the kept-probabilities scratch are larger than the 126 MB L2"
                          % (v * h * 2 / 1e6)},
         "rows_per_s": total_rows * args.steps / (ms_total * 1e-3),
         "executed_tflops": round(step_flops * world / (ms_per_step * 1e-3) / 1e12, 1),
-        "rows_processed": {"fwd": fwd_rows, "bwd": bwd_rows, "of": n},
-        "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "ms_per_step": e2e_ms_total / args.steps},
-        "gpu_launches": int(launches),
-        "clocks": clocks,
+        "rows_processed": {"fwd": n_valid, "bwd": r["bwd_rows"], "of": n},
+        "ms_per_step_with_kernel_events": r["ms_profiled"] / args.steps,
+        "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": r["e2e"]["h2d"],
+                "d2h_bytes_per_step": r["e2e"]["d2h"], "ms_per_step": e2e_ms_total / args.steps,
+                "h2d_ms_per_step": r["e2e"]["h2d_ms"]},
+        "gpu_launches": int(r["launches"]),
+        "clocks": r["clocks"],
         "roofline": roofline,
         "kernels": kernels,
+        "configs": configs,
         "cpu_baseline": cpu_baseline,
-        "loss": float(loss.item()),
+        "loss": r["loss"],
     }
     print(json.dumps(line), flush=True)
     if world > 1:
@@ -436,19 +526,18 @@ def run_ours(args):
 
 
 # ------------------------------------------------------------------------------------ loss-only sweep
-def run_loss_sweep(args):
-    """Loss kernels alone on the bandwidth-sweep workload: fwd, bwd and fused fwd+bwd at --tokens tokens.
-    Every iteration is timed with its own CUDA-event pair; when the inputs are smaller than 2x L2 a 512 MB
-    buffer is overwritten between iterations (untimed) to flush L2."""
+def loss_sweep_entry(n, sampler, dev, peaks, *, min_seconds=1.5, warmup=3):
+    """Loss calls alone on the bandwidth-sweep workload at n tokens: fwd, bwd and fused fwd+bwd.  Each call is
+    timed over a back-to-back loop of at least `min_seconds` (the per-token arrays, 21 n bytes, exceed L2 at
+    both sizes the sweep is judged at; below 2 x L2 a 512 MB buffer is overwritten between iterations instead
+    and every iteration gets its own event pair).  `call` figures cover every launch of the ABI call; `kernel`
+    figures the streaming kernel alone, from the library's per-launch events in a second loop."""
     import numpy as np
     import torch
 
     import paper_2512_06547_b200 as a3po
     from paper_2512_06547_b200 import workloads
 
-    dev = torch.device("cuda", 0)
-    torch.cuda.set_device(dev)
-    n = args.tokens
     inp = workloads.loss_sweep(n)
     to_dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(dev)
     logp, behav, versions, adv, mask = (to_dev(inp[k]) for k in ("logp", "behav_logp", "versions", "adv", "mask"))
@@ -463,78 +552,131 @@ def run_loss_sweep(args):
         "bwd": (lambda: a3po.a3po_loss_bwd(*common, grad, ws, fwd_stats=stats), 21),
         "fwd_bwd": (lambda: a3po.a3po_loss_fwd_bwd(*common, loss, grad, ws, stats=stats), 22),
     }
-    peaks = load_peaks()
-    sampler = ClockSampler(0)
-    sampler.start()
     results = {}
-    a3po.a3po_profile_enable(True)
-    sampler_marked = False
+    t_begin = time.monotonic()
     for name, (fn, bytes_per_token) in calls.items():
-        for _ in range(max(args.warmup, 3)):
+        a3po.a3po_profile_enable(False)
+        for _ in range(max(warmup, 3)):
             fn()
         torch.cuda.synchronize()
-        a3po.a3po_profile_read()
-        if not sampler_marked:
-            sampler.mark_begin()
-            sampler_marked = True
-        call_ms = []
-        for _ in range(args.steps):
-            if flush is not None:
-                flush.fill_(1)
+        est = max(bytes_per_token * n / 5e12, 2e-5)
+        iters = steps_for(est, min_seconds / len(calls), 20, 20000)
+        if flush is None:
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
-            fn()
+            for _ in range(iters):
+                fn()
             e1.record()
             torch.cuda.synchronize()
-            call_ms.append(e0.elapsed_time(e1))
+            call_ms = e0.elapsed_time(e1) / iters
+        else:
+            iters = min(iters, 200)
+            per = []
+            for _ in range(iters):
+                flush.fill_(1)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                fn()
+                e1.record()
+                torch.cuda.synchronize()
+                per.append(e0.elapsed_time(e1))
+            call_ms = statistics.mean(per)
+        # the streaming kernel alone, and the launches of one call
+        a3po.a3po_profile_enable(True)
+        a3po.a3po_profile_read()
+        reps = 20
+        for _ in range(reps):
+            if flush is not None:
+                flush.fill_(1)
+            fn()
+        torch.cuda.synchronize()
+        a3po.a3po_profile_enable(False)
         prof = a3po.a3po_profile_read()
         main_ms = [ms for k, ms in prof if k in ("loss_fwd", "loss_bwd", "loss_fwd_bwd")]
         kernel_ms = statistics.mean(main_ms)
         main_bytes = bytes_per_token - (1 if name == "fwd_bwd" else 0)     # the mask pre-count is its own kernel
         results[name] = {
-            "call_ms": statistics.mean(call_ms), "kernel_ms": kernel_ms, "launches_per_call": len(prof) // args.steps,
-            "algorithmic_bytes_per_token": bytes_per_token,
-            "call_gbs": bytes_per_token * n / (statistics.mean(call_ms) * 1e-3) / 1e9,
-            "kernel_gbs": main_bytes * n / (kernel_ms * 1e-3) / 1e9,
+            "call_ms": round(call_ms, 5), "kernel_ms": round(kernel_ms, 5), "launches_per_call": len(prof) // reps,
+            "iterations": iters, "algorithmic_bytes_per_token": bytes_per_token,
+            "call_gbs": round(bytes_per_token * n / (call_ms * 1e-3) / 1e9, 1),
+            "kernel_gbs": round(main_bytes * n / (kernel_ms * 1e-3) / 1e9, 1),
         }
-    sampler.mark_end()
-    a3po.a3po_profile_enable(False)
-    clocks = sampler.stop()
+    t_end = time.monotonic()
     best = results["fwd_bwd"]
-    line = {
-        "metric": METRIC, "value": n / (best["call_ms"] * 1e-3), "unit": "tokens/s", "n_gpus": 1, "steps": args.steps,
-        "warmup": max(args.warmup, 3), "ms_per_step": best["call_ms"], "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": f"loss-only bandwidth sweep, N={n} tokens: fp32 logp / behaviour logp ~ -Exp(1), int32 "
-                               "per-token versions (staleness U{0..8}), fp32 advantage, uint8 mask (90% kept), eps=0.2",
-                   "l2": "flushed between iterations" if flush is not None else "inputs exceed L2"},
-        "roofline": {"bound": "hbm", "kernel": "loss_fwd_bwd", "achieved": round(best["kernel_gbs"], 1),
-                     "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": round(best["kernel_gbs"] / peaks["hbm_gbs"], 4),
-                     "frac_of_nominal_8000": round(best["kernel_gbs"] / 8000.0, 4),
+    hbm = peaks["hbm_gbs"]
+    entry = {
+        "workload": f"loss-only bandwidth sweep, N={n} tokens: fp32 logp / behaviour logp ~ -Exp(1), int32 per-token "
+                    "versions (staleness U{0..8}), fp32 advantage, uint8 mask (90% kept), eps=0.2",
+        "l2": "flushed between iterations" if flush is not None else "inputs exceed L2",
+        "value": round(n / (best["call_ms"] * 1e-3), 1), "unit": "tokens/s", "ms_per_call": best["call_ms"],
+        "roofline": {"bound": "hbm", "kernel": "a3po_loss_fwd_bwd (whole call, every launch)",
+                     "achieved": best["call_gbs"], "peak": hbm, "unit": "GB/s",
+                     "frac": round(best["call_gbs"] / hbm, 4),
+                     "frac_of_nominal_8000": round(best["call_gbs"] / 8000.0, 4),
+                     "kernel_only_achieved": best["kernel_gbs"], "kernel_only_frac": round(best["kernel_gbs"] / hbm, 4),
                      "traffic": round(NCU_TRAFFIC_PER_TOKEN_LOSS["loss_fwd_bwd"] * n),
-                     "algorithmic_bytes_per_launch": 21 * n,
+                     "algorithmic_bytes_per_call": 22 * n,
                      "peak_source": f"{peaks['_source']} copy bandwidth"},
-        "loss_kernels": results, "clocks": clocks, "gpu_launches": None, "e2e": None, "cpu_baseline": None,
+        "loss_calls": results,
+        "clocks": sampler.window(t_begin, t_end) if sampler else None,
+    }
+    del logp, behav, versions, adv, mask, ws, grad, flush
+    torch.cuda.empty_cache()
+    return entry
+
+
+def run_loss_sweep(args):
+    import torch
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    peaks = load_peaks()
+    sampler = ClockSampler(0)
+    sampler.start()
+    time.sleep(0.3)
+    entry = loss_sweep_entry(args.tokens, sampler, dev, peaks, min_seconds=max(1.5, 0.05 * args.steps),
+                             warmup=args.warmup)
+    sampler.stop()
+    line = {
+        "metric": METRIC, "value": entry["value"], "unit": "tokens/s", "n_gpus": 1, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": entry["ms_per_call"], "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": entry["workload"], "l2": entry["l2"]},
+        "roofline": entry["roofline"], "loss_calls": entry["loss_calls"], "clocks": entry["clocks"],
+        "gpu_launches": None, "e2e": None, "cpu_baseline": None,
     }
     print(json.dumps(line), flush=True)
+
+
+def respawn_under_torchrun(args):
+    """`python bench.py --gpus N` with N > 1 outside torchrun: start one rank per GPU and hand over."""
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="1p5b", choices=sorted(WORKLOAD_TEXT) + ["loss_sweep"])
+    ap.add_argument("--workload", default="8b", choices=sorted(WORKLOAD_TEXT) + ["loss_sweep"])
     ap.add_argument("--tokens", type=int, default=1 << 26, help="token count of --workload loss_sweep")
     ap.add_argument("--oracle-rows", type=int, default=256)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-configs", action="store_true",
+                    help="skip the compact entries for the other named configurations")
     ap.add_argument("--small", action="store_true",
                     help="same shapes with 4 sequences only (a profiler-sized case; not a benchmark number)")
     ap.add_argument("--separate-calls", action="store_true",
                     help="time fwd / loss / bwd as three ABI calls (backward recomputes the logits) instead of "
                          "a3po_train_step")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(respawn_under_torchrun(args))
     if args.workload == "loss_sweep":
         run_loss_sweep(args)
     elif args.impl == "reference":

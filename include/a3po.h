@@ -50,6 +50,9 @@ typedef enum { A3PO_F32 = 0, A3PO_BF16 = 1 } a3po_dtype;
 /* Bits of the optional device status word. */
 #define A3PO_STATUS_TARGET_OUT_OF_RANGE 1u /* some targets[t] was outside [0,V) and was clamped */
 #define A3PO_STATUS_WAIT_TIMEOUT 2u        /* a bounded pipeline wait expired; results invalid  */
+#define A3PO_STATUS_KEPT_RANGE 4u          /* keep-path only: some row's target probability is below
+                                              about 1e-37, beyond what the kept ratios can express;
+                                              that row's gradient contribution was dropped          */
 
 /* Side outputs of the loss forward: the paper's per-step stability diagnostics
  * (importance-weight max/min, Fig. 5; number of clipped tokens, Fig. 6). */
@@ -115,36 +118,43 @@ int a3po_token_logprobs_bwd(const void* hidden, const void* w, const int32_t* ta
                             uint32_t* status, void* stream);
 
 /* --------------------------------------------------------------------------------------------
- * Forward / backward pair that shares the logits instead of recomputing them (bf16 inputs only;
- * no counterpart in the paper).  For callers whose forward and backward are separate calls, as
- * under an autograd engine:
+ * Forward / backward pair that shares the softmax instead of recomputing the logits (bf16 inputs
+ * only; no counterpart in the paper).  For callers whose forward and backward are separate calls,
+ * as under an autograd engine:
  *
- *   a3po_token_logprobs_fwd_keep  = a3po_token_logprobs_fwd (same logp, lse; rows with row_mask 0
- *       are skipped) that also fills `kept` with the logits of the rows that took part: fp16,
- *       shifted by a per-row reference per 256 vocabulary columns so that the entries that matter
- *       for the softmax are stored accurately, plus the references and the row map.
+ *   a3po_token_logprobs_fwd_keep  = a3po_token_logprobs_fwd (same logp, lse, entropy; rows with
+ *       row_mask 0 are skipped) that also fills `kept`.  For each row that took part it keeps the
+ *       probability ratios q[t,v] = exp(z[t,v] - z[t,y_t]) = p[t,v] / p[t,y_t] in bf16 (a float
+ *       ratio keeps bf16's relative precision whether the row is flat or peaked) and their sum
+ *       s[t] over v != y_t, from which lse = z_y + log1p(s), logp = -log1p(s) and
+ *       1 - p_y = s / (1 + s) follow without cancellation.
  *   a3po_token_logprobs_bwd_kept  = a3po_token_logprobs_bwd (same grad_hidden, grad_w within the
- *       gradient tolerance) that turns `kept` into dz in one streaming pass and runs only the two
- *       gradient contractions: 4 N V H flops instead of 6 N V H for the backward.
+ *       gradient tolerance) that runs only the two gradient contractions, directly on q:
+ *       dz[t,v] = a_t q'[t,v] with a_t = -grad_logp[t] inv_T / (1 + s[t]) and q'[t,y_t] = -s[t], so
+ *       grad_hidden = diag(a) (q' W) and grad_w = q'^T (diag(a) hidden): 4 N V H flops instead of
+ *       6 N V H for the backward, and no pass over an [N,V] matrix besides the contractions.
  *
- * `kept`: device buffer of a3po_kept_logits_bytes(N, V) bytes (about 2 N V bytes), 256-byte
- * aligned, written by the forward, read by the backward; hidden, w, targets and lse must be the
- * forward's.  Rows skipped by the forward must have grad_logp == 0.  Both calls return
- * A3PO_ERR_UNSUPPORTED for shapes the tensor-core path does not take (H % 8 != 0): use the plain
- * pair then.  ws: at least the matching *_workspace_bytes.
+ * `kept`: device buffer of a3po_kept_bytes(N, V) bytes (about 2 N V), 256-byte aligned, written by
+ * the forward, read by the backward, which also writes the target entries q'[t,y_t] into it (the
+ * same values on every call, so the backward may be repeated).  hidden, w, targets must be the
+ * forward's; `lse` is accepted for symmetry with a3po_token_logprobs_bwd and not read.  Rows the
+ * forward skipped get a zero gradient whatever their grad_logp.  A row whose target probability
+ * is below about 1e-37 cannot be kept (A3PO_STATUS_KEPT_RANGE is raised, its contribution is
+ * dropped).  Both calls return A3PO_ERR_UNSUPPORTED for shapes the tensor-core path does not take
+ * (H % 8 != 0): use the plain pair then.  ws: at least the matching *_workspace_bytes.
  * ------------------------------------------------------------------------------------------ */
-size_t a3po_kept_logits_bytes(int64_t N, int V);
+size_t a3po_kept_bytes(int64_t N, int V);
 size_t a3po_token_logprobs_fwd_keep_workspace_bytes(int64_t N, int H, int V);
 size_t a3po_token_logprobs_bwd_kept_workspace_bytes(int64_t N, int H, int V);
 
 int a3po_token_logprobs_fwd_keep(const void* hidden, const void* w, const int32_t* targets,
                                  const uint8_t* row_mask, int64_t N, int H, int V,
-                                 float inv_temperature, float* logp, float* lse, void* kept,
-                                 size_t kept_bytes, void* ws, size_t ws_bytes, uint32_t* status,
-                                 void* stream);
+                                 float inv_temperature, float* logp, float* lse, float* entropy,
+                                 void* kept, size_t kept_bytes, void* ws, size_t ws_bytes,
+                                 uint32_t* status, void* stream);
 
 int a3po_token_logprobs_bwd_kept(const void* hidden, const void* w, const int32_t* targets,
-                                 const float* lse, const float* grad_logp, const void* kept,
+                                 const float* lse, const float* grad_logp, void* kept,
                                  size_t kept_bytes, int64_t N, int H, int V, float inv_temperature,
                                  void* grad_hidden, float* grad_w, int accumulate_grad_w, void* ws,
                                  size_t ws_bytes, uint32_t* status, void* stream);
@@ -171,7 +181,8 @@ int a3po_token_logprobs_bwd_kept(const void* hidden, const void* w, const int32_
  *   range [cu_seqlens[b], cu_seqlens[b+1]) with cu_seqlens[0] = 0 and cu_seqlens[B] = N.
  * clip_eps >= 0.
  * loss: fp32 device scalar.  stats: device struct or NULL.
- * The reduction is a fixed two-stage tree: results are bit-identical from run to run.
+ * The reduction is a fixed two-stage tree: results are bit-identical from run to run.  Where the
+ * device supports cooperative launches the whole call is one kernel launch.
  * ws/ws_bytes: at least a3po_loss_workspace_bytes(N).
  * ------------------------------------------------------------------------------------------ */
 size_t a3po_loss_workspace_bytes(int64_t N);
@@ -288,41 +299,46 @@ int a3po_loss_fwd_static(const float* logp, const float* behav_logp, const int32
                          float clip_eps, float* loss, a3po_stats* stats, void* stream);
 
 /* --------------------------------------------------------------------------------------------
- * One whole training-step pass with per-step inputs in HOST memory (no counterpart in the
- * paper; this is the end-to-end form of the four calls above):
- *   copies hidden, targets, behav_logp, versions, adv, mask host->device, runs
- *   token_logprobs_fwd -> loss_fwd_bwd -> token_logprobs_bwd, copies loss + stats back.
+ * One whole training-step pass with every buffer on the device (no counterpart in the paper):
+ *   logp, lse [, entropy]  = token_logprobs_fwd(hidden, w, targets, row_mask = mask)
+ *   loss, stats, grad_logp = loss_fwd_bwd(logp, behav_logp, versions (per token), ...)   detach_prox = 1
+ *   grad_hidden, grad_w    = token_logprobs_bwd(..., lse, grad_logp)
+ * with the same results as the three calls.  For bf16 inputs and a workspace of at least
+ * a3po_train_step_workspace_bytes(...) the step does not recompute the LM head in the backward
+ * (6 N V H flops instead of 8 N V H): the rows with mask != 0 are gathered once (their number M
+ * is then known on the device), and per chunk of those rows the forward keeps the softmax as
+ * bf16 probability ratios (see a3po_token_logprobs_fwd_keep), the loss forward + backward runs
+ * on the chunk's log-probs, and the two gradient contractions run on the kept ratios.  The
+ * workspace holds one chunk of ratios at a time (chunk x V x 2 bytes; the recommended size is
+ * for chunks of 65,536 rows, about 20 GB at V = 151,936, and a larger workspace gives larger
+ * chunks) plus a gathered copy of hidden.  With a smaller workspace (at least
+ * a3po_train_step_min_workspace_bytes) or fp32 inputs the three calls are made as they are.
+ * logp, lse, grad_logp: fp32 [N] outputs.  entropy: fp32 [N] or NULL (policy entropy per row,
+ * Fig. 4).  Other arguments as in the individual calls.
+ * ------------------------------------------------------------------------------------------ */
+size_t a3po_train_step_min_workspace_bytes(int64_t N, int H, int V, a3po_dtype dt);
+size_t a3po_train_step_workspace_bytes(int64_t N, int H, int V, a3po_dtype dt);
+
+int a3po_train_step(const void* hidden, const int32_t* targets, const float* behav_logp,
+                    const int32_t* versions, const float* adv, const uint8_t* mask, int64_t N, int H,
+                    int V, a3po_dtype dt, int32_t current_version, float clip_eps,
+                    float inv_temperature, const void* w, float* grad_w, int accumulate_grad_w,
+                    void* grad_hidden, float* logp, float* lse, float* entropy, float* grad_logp,
+                    float* loss, a3po_stats* stats, void* ws, size_t ws_bytes, uint32_t* status,
+                    void* stream);
+
+/* --------------------------------------------------------------------------------------------
+ * The same pass with per-step inputs in HOST memory (no counterpart in the paper; this is the
+ * end-to-end form of the call above):
+ *   copies hidden, targets, behav_logp, versions, adv, mask host->device, runs a3po_train_step,
+ *   copies loss + stats back.
  * h_* are host pointers (pinned memory recommended; pageable works but serialises).
  * d_w, d_grad_w (accumulated into when accumulate_grad_w != 0), d_grad_hidden ([N,H] dt) and
  * d_stage/d_ws are device buffers.  d_stage needs a3po_train_step_stage_bytes(N,H,dt) bytes and
  * d_ws a3po_train_step_workspace_bytes(N,H,V,dt).  h_loss (float) and h_stats are host outputs,
  * valid after the caller synchronises `stream`.
  * ------------------------------------------------------------------------------------------ */
-/* --------------------------------------------------------------------------------------------
- * One whole training-step pass with every buffer on the device (no counterpart in the paper):
- *   logp, lse   = token_logprobs_fwd(hidden, w, targets, row_mask = mask)
- *   loss, stats, grad_logp = loss_fwd_bwd(logp, behav_logp, versions (per token), ...)   detach_prox = 1
- *   grad_hidden, grad_w    = token_logprobs_bwd(..., lse, grad_logp)
- * with the same results as the three calls.  Given a workspace of
- * a3po_train_step_workspace_bytes(...) and bf16 inputs, the forward keeps its logits (fp16, shifted
- * by a per-row, per-256-column reference so that the entries that matter are stored accurately;
- * rows with mask != 0 only) and the backward builds dz from them in one streaming pass instead of
- * recomputing the LM head: 6 N V H flops per step instead of 8 N V H.  The kept logits live in the
- * workspace only (N_valid x V x 2 bytes).  With a smaller workspace (at least
- * a3po_train_step_min_workspace_bytes) the three calls are made as they are.
- * logp, lse, grad_logp: fp32 [N] outputs.  Other arguments as in the individual calls.
- * ------------------------------------------------------------------------------------------ */
-size_t a3po_train_step_min_workspace_bytes(int64_t N, int H, int V, a3po_dtype dt);
-
-int a3po_train_step(const void* hidden, const int32_t* targets, const float* behav_logp,
-                    const int32_t* versions, const float* adv, const uint8_t* mask, int64_t N, int H,
-                    int V, a3po_dtype dt, int32_t current_version, float clip_eps,
-                    float inv_temperature, const void* w, float* grad_w, int accumulate_grad_w,
-                    void* grad_hidden, float* logp, float* lse, float* grad_logp, float* loss,
-                    a3po_stats* stats, void* ws, size_t ws_bytes, uint32_t* status, void* stream);
-
 size_t a3po_train_step_stage_bytes(int64_t N, int H, a3po_dtype dt);
-size_t a3po_train_step_workspace_bytes(int64_t N, int H, int V, a3po_dtype dt);
 
 int a3po_train_step_host(const void* h_hidden, const int32_t* h_targets, const float* h_behav_logp,
                          const int32_t* h_versions, const float* h_adv, const uint8_t* h_mask,

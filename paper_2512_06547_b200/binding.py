@@ -19,6 +19,7 @@ A3PO_F32 = 0
 A3PO_BF16 = 1
 STATUS_TARGET_OUT_OF_RANGE = 1
 STATUS_WAIT_TIMEOUT = 2
+STATUS_KEPT_RANGE = 4
 
 
 class A3poStats(ctypes.Structure):
@@ -62,19 +63,19 @@ _SIGNATURES = {
     "a3po_grpo_advantages": (c_int, [c_void_p, c_int, c_int, c_void_p, c_int64, c_float, c_void_p, c_void_p, c_size_t,
                                      c_void_p]),
     "a3po_selftest_wait_timeout": (c_int, [c_void_p, ctypes.c_uint, c_void_p]),
-    "a3po_kept_logits_bytes": (c_size_t, [c_int64, c_int]),
+    "a3po_kept_bytes": (c_size_t, [c_int64, c_int]),
     "a3po_token_logprobs_fwd_keep_workspace_bytes": (c_size_t, [c_int64, c_int, c_int]),
     "a3po_token_logprobs_bwd_kept_workspace_bytes": (c_size_t, [c_int64, c_int, c_int]),
     "a3po_token_logprobs_fwd_keep": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_int, c_int, c_float,
-                                             c_void_p, c_void_p, c_void_p, c_size_t, c_void_p, c_size_t, c_void_p,
-                                             c_void_p]),
+                                             c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p, c_size_t,
+                                             c_void_p, c_void_p]),
     "a3po_token_logprobs_bwd_kept": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t,
                                              c_int64, c_int, c_int, c_float, c_void_p, c_void_p, c_int, c_void_p,
                                              c_size_t, c_void_p, c_void_p]),
     "a3po_train_step_min_workspace_bytes": (c_size_t, [c_int64, c_int, c_int, c_int]),
     "a3po_train_step": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_int, c_int, c_int,
                                 c_int32, c_float, c_float, c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_void_p,
-                                c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p, c_void_p]),
+                                c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p, c_void_p]),
     "a3po_train_step_host": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_int, c_int,
                                      c_int, c_int32, c_float, c_float, c_void_p, c_void_p, c_int, c_void_p, c_void_p,
                                      c_size_t, c_void_p, c_size_t, c_void_p, c_void_p, c_void_p, c_void_p]),
@@ -220,8 +221,8 @@ def a3po_token_logprobs_bwd(hidden, w, targets, lse, grad_logp, grad_hidden, gra
     _check("a3po_token_logprobs_bwd", rc)
 
 
-def a3po_kept_logits_bytes(N, V) -> int:
-    return load_library().a3po_kept_logits_bytes(N, V)
+def a3po_kept_bytes(N, V) -> int:
+    return load_library().a3po_kept_bytes(N, V)
 
 
 def a3po_token_logprobs_fwd_keep_workspace_bytes(N, H, V) -> int:
@@ -232,26 +233,27 @@ def a3po_token_logprobs_bwd_kept_workspace_bytes(N, H, V) -> int:
     return load_library().a3po_token_logprobs_bwd_kept_workspace_bytes(N, H, V)
 
 
-def a3po_token_logprobs_fwd_keep(hidden, w, targets, logp, lse, kept, ws, *, row_mask=None, inv_temperature=1.0,
-                                 status=None, stream=None):
-    """Forward that also fills `kept` (uint8 buffer of a3po_kept_logits_bytes) for a3po_token_logprobs_bwd_kept."""
+def a3po_token_logprobs_fwd_keep(hidden, w, targets, logp, lse, kept, ws, *, row_mask=None, entropy=None,
+                                 inv_temperature=1.0, status=None, stream=None):
+    """Forward that also fills `kept` (uint8 buffer of a3po_kept_bytes) for a3po_token_logprobs_bwd_kept."""
     _want(hidden, torch.bfloat16, "hidden"); _want(w, torch.bfloat16, "w")
     _want(targets, torch.int32, "targets"); _want(row_mask, torch.uint8, "row_mask")
-    _want(logp, torch.float32, "logp"); _want(lse, torch.float32, "lse")
+    _want(logp, torch.float32, "logp"); _want(lse, torch.float32, "lse"); _want(entropy, torch.float32, "entropy")
     _want(kept, torch.uint8, "kept"); _want(ws, torch.uint8, "ws"); _want(status, torch.int32, "status")
     n, h = hidden.shape
     v = w.shape[0]
     if w.shape[1] != h or targets.numel() != n or logp.numel() != n or lse.numel() != n:
         raise ValueError("shape mismatch")
     rc = load_library().a3po_token_logprobs_fwd_keep(_ptr(hidden), _ptr(w), _ptr(targets), _ptr(row_mask), n, h, v,
-                                                     float(inv_temperature), _ptr(logp), _ptr(lse), _ptr(kept),
-                                                     kept.numel(), _ptr(ws), ws.numel(), _ptr(status), _stream(stream))
+                                                     float(inv_temperature), _ptr(logp), _ptr(lse), _ptr(entropy),
+                                                     _ptr(kept), kept.numel(), _ptr(ws), ws.numel(), _ptr(status),
+                                                     _stream(stream))
     _check("a3po_token_logprobs_fwd_keep", rc)
 
 
 def a3po_token_logprobs_bwd_kept(hidden, w, targets, lse, grad_logp, kept, grad_hidden, grad_w, ws, *,
                                  accumulate_grad_w=False, inv_temperature=1.0, status=None, stream=None):
-    """Backward from the logits kept by a3po_token_logprobs_fwd_keep (no recomputation of the LM head)."""
+    """Backward from what a3po_token_logprobs_fwd_keep kept (no recomputation of the LM head)."""
     _want(hidden, torch.bfloat16, "hidden"); _want(w, torch.bfloat16, "w")
     _want(grad_hidden, torch.bfloat16, "grad_hidden"); _want(targets, torch.int32, "targets")
     _want(lse, torch.float32, "lse"); _want(grad_logp, torch.float32, "grad_logp")
@@ -390,10 +392,10 @@ def a3po_train_step_min_workspace_bytes(N, H, V, dt) -> int:
 
 
 def a3po_train_step(hidden, w, targets, behav_logp, versions, current_version, adv, mask, clip_eps, logp, lse,
-                    grad_logp, loss, grad_hidden, grad_w, ws, *, stats=None, accumulate_grad_w=False,
+                    grad_logp, loss, grad_hidden, grad_w, ws, *, stats=None, entropy=None, accumulate_grad_w=False,
                     inv_temperature=1.0, status=None, stream=None):
     """token_logprobs_fwd -> loss_fwd_bwd -> token_logprobs_bwd in one call; with the recommended workspace the
-    backward reuses logits kept by the forward instead of recomputing them."""
+    backward reuses the softmax kept by the forward instead of recomputing the logits."""
     dt = _dtype_code(hidden)
     _want(hidden, hidden.dtype, "hidden"); _want(w, hidden.dtype, "w"); _want(grad_hidden, hidden.dtype, "grad_hidden")
     _want(targets, torch.int32, "targets"); _want(versions, torch.int32, "versions"); _want(mask, torch.uint8, "mask")
@@ -401,18 +403,20 @@ def a3po_train_step(hidden, w, targets, behav_logp, versions, current_version, a
                   (loss, "loss"), (grad_w, "grad_w")):
         _want(t, torch.float32, nm)
     _want(stats, torch.uint8, "stats"); _want(status, torch.int32, "status"); _want(ws, torch.uint8, "ws")
+    _want(entropy, torch.float32, "entropy")
     n, h = hidden.shape
     v = w.shape[0]
     if w.shape[1] != h or grad_w.shape != w.shape or grad_hidden.shape != hidden.shape:
         raise ValueError("shape mismatch")
-    for t in (targets, behav_logp, versions, adv, mask, logp, lse, grad_logp):
+    for t in (targets, behav_logp, versions, adv, mask, logp, lse, grad_logp) + ((entropy,) if entropy is not None
+                                                                                  else ()):
         if t.numel() != n:
             raise ValueError("per-token arrays must have N entries")
     rc = load_library().a3po_train_step(
         _ptr(hidden), _ptr(targets), _ptr(behav_logp), _ptr(versions), _ptr(adv), _ptr(mask), n, h, v, dt,
         int(current_version), float(clip_eps), float(inv_temperature), _ptr(w), _ptr(grad_w),
-        int(bool(accumulate_grad_w)), _ptr(grad_hidden), _ptr(logp), _ptr(lse), _ptr(grad_logp), _ptr(loss),
-        _ptr(stats), _ptr(ws), ws.numel(), _ptr(status), _stream(stream))
+        int(bool(accumulate_grad_w)), _ptr(grad_hidden), _ptr(logp), _ptr(lse), _ptr(entropy), _ptr(grad_logp),
+        _ptr(loss), _ptr(stats), _ptr(ws), ws.numel(), _ptr(status), _stream(stream))
     _check("a3po_train_step", rc)
 
 

@@ -30,15 +30,16 @@ int sm_count();
 enum KernelId : int {
   kKLossFwd = 0, kKLossBwd, kKLossFwdBwd, kKLossFinalize, kKMaskCount, kKMaskCountFinalize, kKExpandVersions,
   kKMergePartials, kKSimtFwd, kKSimtDz, kKSimtGemm, kKTcFwd, kKTcDz, kKTcGradHidden, kKTcGradW, kKCompact, kKGrpo,
-  kKSelfTest, kKTcFwdSave, kKDzSaved,
+  kKSelfTest, kKTcFwdKeep, kKKeptRows, kKH2D,
   kKernelIdCount
 };
 
 // When profiling is enabled (a3po_profile_enable), brackets one kernel launch with a pair of CUDA
 // events recorded on the launch stream; otherwise does nothing.
 struct ProfileScope {
-  int slot;
+  int kernel_id;
   cudaStream_t stream;
+  cudaEvent_t start, stop;  // both null when profiling is off
   ProfileScope(int kernel_id, cudaStream_t s);
   ~ProfileScope();
 };

@@ -1,6 +1,5 @@
 // C ABI of the LM-head log-prob calls, the whole-step host entry and library-wide helpers.
 
-#include <cstdlib>
 #include <cstring>
 #include <mutex>
 #include <vector>
@@ -38,20 +37,30 @@ cudaEvent_t take_event() {
 }
 }  // namespace
 
-ProfileScope::ProfileScope(int kernel_id, cudaStream_t s) : slot(-1), stream(s) {
+// The scope owns its two events until the launch has been bracketed; only then does the finished
+// record enter the list, so a concurrent a3po_profile_read never sees (or recycles) half a record.
+ProfileScope::ProfileScope(int id, cudaStream_t s) : kernel_id(id), stream(s), start(nullptr), stop(nullptr) {
   if (!g_profile_on.load(std::memory_order_relaxed)) return;
-  std::lock_guard<std::mutex> lock(g_profile_mu);
-  ProfileRecord r{kernel_id, take_event(), take_event()};
-  if (!r.start || !r.stop) return;
-  cudaEventRecord(r.start, stream);
-  g_profile_records.push_back(r);
-  slot = static_cast<int>(g_profile_records.size()) - 1;
+  {
+    std::lock_guard<std::mutex> lock(g_profile_mu);
+    start = take_event();
+    stop = take_event();
+  }
+  if (!start || !stop) {
+    std::lock_guard<std::mutex> lock(g_profile_mu);
+    if (start) g_event_pool.push_back(start);
+    if (stop) g_event_pool.push_back(stop);
+    start = stop = nullptr;
+    return;
+  }
+  cudaEventRecord(start, stream);
 }
 
 ProfileScope::~ProfileScope() {
-  if (slot < 0) return;
+  if (!start) return;
+  cudaEventRecord(stop, stream);
   std::lock_guard<std::mutex> lock(g_profile_mu);
-  if (slot < static_cast<int>(g_profile_records.size())) cudaEventRecord(g_profile_records[slot].stop, stream);
+  g_profile_records.push_back(ProfileRecord{kernel_id, start, stop});
 }
 
 int sm_count() {
@@ -117,10 +126,29 @@ merge_partials_kernel(const SoftmaxPartial* __restrict__ part, const float* __re
   if (entropy) entropy[t] = l - e / s;
 }
 
+// ORs A3PO_STATUS_TARGET_OUT_OF_RANGE into *status if any target lies outside [0, v).
+__global__ void __launch_bounds__(kMergeThreads)
+flag_bad_targets_kernel(const int32_t* __restrict__ targets, long long n, int v, uint32_t* status) {
+  const long long t = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (t >= n) return;
+  const int y = targets[t];
+  if (y < 0 || y >= v) atomicOr(status, A3PO_STATUS_TARGET_OUT_OF_RANGE);
+}
+
+int flag_bad_targets(const int32_t* targets, long long n, int v, uint32_t* status, cudaStream_t stream) {
+  if (!status || n <= 0) return A3PO_OK;
+  const unsigned blocks = static_cast<unsigned>((n + kMergeThreads - 1) / kMergeThreads);
+  A3PO_LAUNCH(kKMergePartials, stream, (flag_bad_targets_kernel<<<blocks, kMergeThreads, 0, stream>>>(targets, n, v,
+                                                                                                      status)));
+  return after_launch();
+}
+
 int simt_fwd_splits(long long n, int v) {
   const long long row_tiles = (n + kSimtTile - 1) / kSimtTile;
   const int n_tiles = (v + kSimtTile - 1) / kSimtTile;
-  long long s = row_tiles > 0 ? (148 * 4 + row_tiles - 1) / row_tiles : 1;
+  int sms = sm_count();
+  if (sms <= 0) sms = 148;
+  long long s = row_tiles > 0 ? (static_cast<long long>(sms) * 4 + row_tiles - 1) / row_tiles : 1;
   if (s > n_tiles) s = n_tiles;
   if (s > 64) s = 64;
   if (s < 1) s = 1;
@@ -133,15 +161,8 @@ size_t fwd_ws_for(long long n, int splits) {
          round_up(rows * sizeof(float), 256) + 256;
 }
 
-bool env_flag(const char* name) {
-  const char* e = std::getenv(name);
-  return e && e[0] == '1';
-}
-
-bool force_simt() { return env_flag("A3PO_FORCE_SIMT"); }
-
 bool use_tc(a3po_dtype dt, const void* hidden, const void* w, long long n, int h, int v) {
-  return dt == A3PO_BF16 && !force_simt() && lmhead_tc_supported(hidden, w, n, h, v);
+  return dt == A3PO_BF16 && lmhead_tc_supported(hidden, w, n, h, v);
 }
 
 size_t elt_size(a3po_dtype dt) { return dt == A3PO_F32 ? 4 : 2; }
@@ -188,7 +209,7 @@ const char* a3po_status_string(int code) {
   }
 }
 
-int a3po_version(void) { return 1001; }
+int a3po_version(void) { return 2000; }
 
 int a3po_selftest_wait_timeout(uint32_t* status, unsigned timeout_ms, void* stream) {
   if (!status || timeout_ms == 0 || timeout_ms > 2000) return A3PO_ERR_INVALID_ARG;
@@ -203,7 +224,7 @@ const char* a3po_kernel_name(int kernel_id) {
       "loss_fwd", "loss_bwd", "loss_fwd_bwd", "loss_finalize", "mask_count", "mask_count_finalize",
       "expand_versions", "merge_partials", "lmhead_fwd_fp32pipe", "lmhead_dz_fp32pipe", "gemm_fp32pipe",
       "gemm_tn<fwd_logsoftmax>", "gemm_tn<dz>", "gemm_tn<grad_hidden>", "gemm_tn<grad_w>", "compact_rows", "grpo_advantages", "selftest",
-      "gemm_tn<fwd_logsoftmax+keep_logits>", "dz_from_kept_logits"};
+      "gemm_tn<fwd_logsoftmax+keep>", "kept_rows", "h2d_copies"};
   return (kernel_id >= 0 && kernel_id < kKernelIdCount) ? names[kernel_id] : "?";
 }
 
@@ -386,70 +407,113 @@ size_t a3po_train_step_stage_bytes(int64_t N, int H, a3po_dtype dt) {
 }
 
 // ------------------------------------------------------------------------------------------------
-// Forward that keeps its logits / backward that uses them (no recomputation of the LM head).
+// Forward that keeps its softmax / backward that uses it (no recomputation of the LM head).
 // ------------------------------------------------------------------------------------------------
 namespace {
-// `kept` buffer: pos[N] (row of the batch -> row of the kept logits, -1 for rows that took no part), then the
-// kept logits proper (fp16 u and fp32 references, see lmhead_tc_saved_logits_bytes).
-size_t kept_pos_bytes(long long n) { return round_up(sizeof(int) * static_cast<size_t>(n > 0 ? n : 0), 256); }
+// `kept` buffer: what the backward needs from the forward, all in the compact row space of the rows that took
+// part: their number, the maps batch row <-> compact row, targets, the tail sums s, and the probability ratios q.
+struct KeptLayout {
+  size_t count, pos, idx, targets, sprime, q, total;
+};
+KeptLayout kept_layout(long long n, int v) {
+  KeptLayout k;
+  size_t off = 0;
+  const size_t rows = static_cast<size_t>(n > 0 ? n : 0);
+  const size_t cap = static_cast<size_t>(compact_capacity(n > 0 ? n : 0));
+  auto take = [&](size_t bytes) { size_t o = off; off = round_up(off + bytes, 256); return o; };
+  k.count = take(sizeof(int));
+  k.pos = take(sizeof(int) * rows);
+  k.idx = take(sizeof(int) * cap);
+  k.targets = take(sizeof(int32_t) * cap);
+  k.sprime = take(sizeof(float) * cap);
+  k.q = take(lmhead_tc_kept_bytes(static_cast<long long>(cap), v));
+  k.total = off;
+  return k;
+}
+
+constexpr size_t kScanBytes = 2 * 4096 * sizeof(int);  // block counts + offsets of the compaction scan
+
+size_t fwd_keep_ws_bytes(long long n, int h, int v) {
+  const size_t cap = static_cast<size_t>(compact_capacity(n));
+  const int splits = lmhead_tc_fwd_splits(static_cast<long long>(cap), v);
+  return round_up(kScanBytes, 256) + round_up(cap * static_cast<size_t>(h) * 2, 256) /*hidden_c*/ +
+         4 * round_up(sizeof(float) * cap, 256) /*zy, logp_c, lse_c, ent_c*/ +
+         2 * round_up(sizeof(float) * cap * splits, 256) /*part_s, part_e*/ + 256;
+}
+
+size_t bwd_kept_ws_bytes(long long n, int h) {
+  const size_t cap = static_cast<size_t>(compact_capacity(n));
+  return round_up(sizeof(float) * cap, 256) /*row_scale*/ + 2 * round_up(cap * static_cast<size_t>(h) * 2, 256) + 256;
+}
 }  // namespace
 
-size_t a3po_kept_logits_bytes(int64_t N, int V) {
+size_t a3po_kept_bytes(int64_t N, int V) {
   if (N < 0 || V <= 0) return 0;
-  return kept_pos_bytes(N) + lmhead_tc_saved_logits_bytes(N, V) + 256;
+  return kept_layout(N, V).total + 256;
 }
 
 size_t a3po_token_logprobs_fwd_keep_workspace_bytes(int64_t N, int H, int V) {
   if (N < 0 || H <= 0 || V <= 0) return 0;
-  return compact_ws_bytes(N, H, false) + fwd_ws_for(N, lmhead_tc_fwd_splits(N, V)) + 256;
+  return fwd_keep_ws_bytes(N, H, V);
 }
 
 size_t a3po_token_logprobs_bwd_kept_workspace_bytes(int64_t N, int H, int V) {
   if (N < 0 || H <= 0 || V <= 0) return 0;
-  return compact_ws_bytes(N, H, true) + lmhead_tc_bwd_ws_bytes(compact_capacity(N), N, H, V) + 256;
+  return bwd_kept_ws_bytes(N, H);
 }
 
 int a3po_token_logprobs_fwd_keep(const void* hidden, const void* w, const int32_t* targets, const uint8_t* row_mask,
-                                 int64_t N, int H, int V, float inv_temperature, float* logp, float* lse, void* kept,
-                                 size_t kept_bytes, void* ws, size_t ws_bytes, uint32_t* status, void* stream_) {
+                                 int64_t N, int H, int V, float inv_temperature, float* logp, float* lse,
+                                 float* entropy, void* kept, size_t kept_bytes, void* ws, size_t ws_bytes,
+                                 uint32_t* status, void* stream_) {
   A3PO_RETURN_IF(check_lmhead_args(hidden, w, targets, N, H, V, A3PO_BF16, inv_temperature));
   if (N > 0 && (!logp || !lse)) return A3PO_ERR_INVALID_ARG;
   if (N == 0) return A3PO_OK;
   if (!use_tc(A3PO_BF16, hidden, w, N, H, V)) return A3PO_ERR_UNSUPPORTED;
-  if (!kept || !aligned_to(kept, 256) || kept_bytes < a3po_kept_logits_bytes(N, V)) return A3PO_ERR_WORKSPACE;
-  if (!ws || !aligned_to(ws, 256) || ws_bytes < a3po_token_logprobs_fwd_keep_workspace_bytes(N, H, V))
-    return A3PO_ERR_WORKSPACE;
+  if (!kept || !aligned_to(kept, 256) || kept_bytes < a3po_kept_bytes(N, V)) return A3PO_ERR_WORKSPACE;
+  if (!ws || !aligned_to(ws, 256) || ws_bytes < fwd_keep_ws_bytes(N, H, V)) return A3PO_ERR_WORKSPACE;
   cudaStream_t stream = as_stream(stream_);
-  const int splits = lmhead_tc_fwd_splits(N, V);
+  const KeptLayout kl = kept_layout(N, V);
+  char* kb = static_cast<char*>(kept);
+  const long long cap = compact_capacity(N);
+  const int splits = lmhead_tc_fwd_splits(cap, V);
+
+  Arena arena(ws, ws_bytes);
   CompactBuffers cb;
-  size_t used = 0;
-  if (!compact_carve(ws, ws_bytes, N, H, false, &cb, &used)) return A3PO_ERR_WORKSPACE;
-  Arena arena(static_cast<char*>(ws) + used, ws_bytes - used);
-  SoftmaxPartial* part = arena.take<SoftmaxPartial>(static_cast<size_t>(N) * splits);
-  float* zy = arena.take<float>(static_cast<size_t>(N));
+  cb.cap = cap;
+  cb.count = reinterpret_cast<int*>(kb + kl.count);
+  cb.pos = reinterpret_cast<int*>(kb + kl.pos);
+  cb.idx = reinterpret_cast<int*>(kb + kl.idx);
+  cb.targets_c = reinterpret_cast<int32_t*>(kb + kl.targets);
+  cb.block_counts = arena.take<int>(4096);
+  cb.block_offsets = arena.take<int>(4096);
+  cb.hidden_c = arena.take<__nv_bfloat16>(static_cast<size_t>(cap) * H);
+  cb.lse_c = nullptr;
+  cb.g_c = nullptr;
+  cb.grad_hidden_c = nullptr;
+  float* zy = arena.take<float>(static_cast<size_t>(cap));
+  float* logp_c = arena.take<float>(static_cast<size_t>(cap));
+  float* lse_c = arena.take<float>(static_cast<size_t>(cap));
+  float* ent_c = arena.take<float>(static_cast<size_t>(cap));
+  float* part_s = arena.take<float>(static_cast<size_t>(cap) * splits);
+  float* part_e = arena.take<float>(static_cast<size_t>(cap) * splits);
   if (!arena.ok()) return A3PO_ERR_WORKSPACE;
-  int* kept_pos = static_cast<int*>(kept);
-  void* saved = static_cast<char*>(kept) + kept_pos_bytes(N);
+  float* sprime = reinterpret_cast<float*>(kb + kl.sprime);
+  void* q = kb + kl.q;
 
   A3PO_RETURN_IF(compact_rows(hidden, H, targets, row_mask, nullptr, nullptr, N, cb, stream));
-  A3PO_RETURN_IF(lmhead_fwd_save_tc(cb.hidden_c, w, cb.targets_c, N, H, V, inv_temperature, splits, part, zy, saved,
-                                    cb.count, status, stream));
-  const unsigned blocks = static_cast<unsigned>((N + kMergeThreads - 1) / kMergeThreads);
-  A3PO_LAUNCH(kKMergePartials, stream, (merge_partials_kernel<<<blocks, kMergeThreads, 0, stream>>>(
-                                           part, nullptr, zy, targets, row_mask, cb.pos, N, V, splits, logp, lse,
-                                           nullptr, status)));
-  A3PO_RETURN_IF(after_launch());
-  // the row map outlives the workspace: the backward finds each row's kept logits through it
-  if (cudaMemcpyAsync(kept_pos, cb.pos, sizeof(int) * static_cast<size_t>(N), cudaMemcpyDeviceToDevice, stream) !=
-      cudaSuccess) {
-    cudaGetLastError();
-    return A3PO_ERR_CUDA;
-  }
-  return A3PO_OK;
+  A3PO_RETURN_IF(target_logits(cb.hidden_c, w, cb.targets_c, cb.count, 0, cap, H, V, inv_temperature, zy, stream));
+  A3PO_RETURN_IF(lmhead_fwd_keep_tc(cb.hidden_c, w, cb.targets_c, zy, cap, H, V, inv_temperature, splits, part_s,
+                                    entropy ? part_e : nullptr, q, cb.count, 0, status, stream));
+  A3PO_RETURN_IF(merge_kept(part_s, part_e, zy, cb.count, 0, cap, splits, inv_temperature, sprime, logp_c, lse_c,
+                            entropy ? ent_c : nullptr, status, stream));
+  A3PO_RETURN_IF(flag_bad_targets(targets, N, V, status, stream));
+  return finish_batch_outputs(cb.pos, N, logp_c, logp, lse_c, lse, nullptr, nullptr, ent_c, entropy, nullptr, H,
+                              stream);
 }
 
 int a3po_token_logprobs_bwd_kept(const void* hidden, const void* w, const int32_t* targets, const float* lse,
-                                 const float* grad_logp, const void* kept, size_t kept_bytes, int64_t N, int H, int V,
+                                 const float* grad_logp, void* kept, size_t kept_bytes, int64_t N, int H, int V,
                                  float inv_temperature, void* grad_hidden, float* grad_w, int accumulate_grad_w,
                                  void* ws, size_t ws_bytes, uint32_t* status, void* stream_) {
   A3PO_RETURN_IF(check_lmhead_args(hidden, w, targets, N, H, V, A3PO_BF16, inv_temperature));
@@ -464,44 +528,89 @@ int a3po_token_logprobs_bwd_kept(const void* hidden, const void* w, const int32_
     return A3PO_OK;
   }
   if (!use_tc(A3PO_BF16, hidden, w, N, H, V)) return A3PO_ERR_UNSUPPORTED;
-  if (!kept || !aligned_to(kept, 256) || kept_bytes < a3po_kept_logits_bytes(N, V)) return A3PO_ERR_WORKSPACE;
-  if (!ws || !aligned_to(ws, 256) || ws_bytes < a3po_token_logprobs_bwd_kept_workspace_bytes(N, H, V))
-    return A3PO_ERR_WORKSPACE;
+  if (!kept || !aligned_to(kept, 256) || kept_bytes < a3po_kept_bytes(N, V)) return A3PO_ERR_WORKSPACE;
+  if (!ws || !aligned_to(ws, 256) || ws_bytes < bwd_kept_ws_bytes(N, H)) return A3PO_ERR_WORKSPACE;
   cudaStream_t stream = as_stream(stream_);
-  CompactBuffers cb;
-  size_t used = 0;
-  if (!compact_carve(ws, ws_bytes, N, H, true, &cb, &used)) return A3PO_ERR_WORKSPACE;
-  void* dz = static_cast<char*>(ws) + used;
-  if (ws_bytes - used < lmhead_tc_bwd_ws_bytes(compact_capacity(N), N, H, V)) return A3PO_ERR_WORKSPACE;
-  const int* kept_pos = static_cast<const int*>(kept);
-  const void* saved = static_cast<const char*>(kept) + kept_pos_bytes(N);
+  const KeptLayout kl = kept_layout(N, V);
+  char* kb = static_cast<char*>(kept);
+  const long long cap = compact_capacity(N);
+  const int* count = reinterpret_cast<const int*>(kb + kl.count);
+  const int* pos = reinterpret_cast<const int*>(kb + kl.pos);
+  const int* idx = reinterpret_cast<const int*>(kb + kl.idx);
+  const int32_t* targets_c = reinterpret_cast<const int32_t*>(kb + kl.targets);
+  const float* sprime = reinterpret_cast<const float*>(kb + kl.sprime);
+  void* q = kb + kl.q;
+  Arena arena(ws, ws_bytes);
+  float* row_scale = arena.take<float>(static_cast<size_t>(cap));
+  __nv_bfloat16* hs = arena.take<__nv_bfloat16>(static_cast<size_t>(cap) * H);
+  __nv_bfloat16* ghc = arena.take<__nv_bfloat16>(static_cast<size_t>(cap) * H);
+  if (!arena.ok()) return A3PO_ERR_WORKSPACE;
 
-  // rows with a non-zero upstream gradient only; dz from the kept logits, then the two contractions
-  A3PO_RETURN_IF(compact_rows(hidden, H, targets, nullptr, grad_logp, lse, N, cb, stream));
-  A3PO_RETURN_IF(dz_from_saved(saved, N, V, kept_pos, cb, inv_temperature, dz, stream));
-  A3PO_RETURN_IF(lmhead_bwd_from_dz_tc(cb.hidden_c, w, dz, N, H, V, cb.grad_hidden_c, grad_w, accumulate_grad_w,
-                                       cb.count, status, stream));
-  return scatter_rows(cb.grad_hidden_c, H, cb.pos, N, grad_hidden, stream);
+  // the target's entry of q and the per-row factor of dz, then the two contractions on q itself
+  A3PO_RETURN_IF(prepare_kept_backward(count, 0, cap, H, V, inv_temperature, sprime, targets_c, nullptr, grad_logp,
+                                       idx, nullptr, hidden, row_scale, q, hs, stream));
+  A3PO_RETURN_IF(lmhead_grad_hidden_from_kept_tc(q, w, row_scale, cap, H, V, ghc, count, 0, status, stream));
+  A3PO_RETURN_IF(scatter_rows(ghc, H, pos, N, grad_hidden, stream));
+  return lmhead_grad_w_from_kept_tc(q, hs, cap, H, V, grad_w, accumulate_grad_w, accumulate_grad_w ? 0 : 1, count, 0,
+                                    status, stream);
 }
 
+// ------------------------------------------------------------------------------------------------
+// Whole step in one call.
+// ------------------------------------------------------------------------------------------------
 namespace {
-// Workspace of the step that keeps the forward's logits (fp16, shifted) for the backward.
-struct SavedStepLayout {
-  size_t kept, kept_bytes, call_ws, call_ws_bytes, loss, total;
+constexpr long long kStepChunkRows = 65536;     // rows of kept ratios the recommended workspace holds at a time
+constexpr long long kStepMinChunkRows = 2048;   // below this the recomputing calls are used instead
+constexpr int kStepMaxSplits = 64;
+
+// Workspace of the step that keeps the forward's softmax for the backward, one chunk of compact rows at a time.
+struct StepLayout {
+  // whole batch
+  size_t count, scan, pos, idx, targets_c, hidden_c, zy, sprime, logp_c, lse_c, g_c, ent_c, behav_c, adv_c, row_scale,
+      versions_c, mask_c, n_valid, partials;
+  // one chunk
+  size_t part_s, part_e, q, hs, ghc;
+  size_t total;
 };
-SavedStepLayout saved_step_layout(long long n, int h, int v) {
-  SavedStepLayout s;
+StepLayout step_layout(long long n, int h, int v, long long chunk_rows) {
+  StepLayout s;
   size_t off = 0;
+  const size_t rows = static_cast<size_t>(n);
+  const size_t cap = static_cast<size_t>(compact_capacity(n));
+  const size_t rc = static_cast<size_t>(chunk_rows);
   auto take = [&](size_t bytes) { size_t o = off; off = round_up(off + bytes, 256); return o; };
-  s.kept_bytes = a3po_kept_logits_bytes(n, v);
-  s.kept = take(s.kept_bytes);
-  const size_t f = a3po_token_logprobs_fwd_keep_workspace_bytes(n, h, v);
-  const size_t b = a3po_token_logprobs_bwd_kept_workspace_bytes(n, h, v);
-  s.call_ws_bytes = f > b ? f : b;   // the forward's and the backward's scratch are never live together
-  s.call_ws = take(s.call_ws_bytes);
-  s.loss = take(a3po_loss_workspace_bytes(n));
+  s.count = take(sizeof(int));
+  s.scan = take(kScanBytes);
+  s.pos = take(4 * rows);
+  s.idx = take(4 * cap);
+  s.targets_c = take(4 * cap);
+  s.hidden_c = take(cap * static_cast<size_t>(h) * 2);
+  s.zy = take(4 * cap); s.sprime = take(4 * cap); s.logp_c = take(4 * cap); s.lse_c = take(4 * cap);
+  s.g_c = take(4 * cap); s.ent_c = take(4 * cap); s.behav_c = take(4 * cap); s.adv_c = take(4 * cap);
+  s.row_scale = take(4 * cap); s.versions_c = take(4 * cap);
+  s.mask_c = take(cap);
+  s.n_valid = take(sizeof(long long));
+  s.partials = take(loss_partial_bytes() * loss_max_partials());
+  s.part_s = take(4 * rc * kStepMaxSplits);
+  s.part_e = take(4 * rc * kStepMaxSplits);
+  s.q = take(lmhead_tc_kept_bytes(chunk_rows, v));
+  s.hs = take(rc * static_cast<size_t>(h) * 2);
+  s.ghc = take(rc * static_cast<size_t>(h) * 2);
   s.total = off;
   return s;
+}
+// Largest chunk (multiple of 128 rows, at most the compact capacity) whose scratch fits `ws_bytes`; 0 if the
+// keeping path does not fit.
+long long step_chunk_rows_for(size_t ws_bytes, long long n, int h, int v) {
+  const long long cap = compact_capacity(n);
+  const size_t fixed = step_layout(n, h, v, 0).total;
+  if (ws_bytes <= fixed) return 0;
+  const size_t per_128 = step_layout(n, h, v, 128).total - fixed;
+  long long rc = static_cast<long long>((ws_bytes - fixed) / per_128) * 128;
+  if (rc > cap) rc = cap;
+  while (rc > 0 && step_layout(n, h, v, rc).total > ws_bytes) rc -= 128;
+  const long long need = cap < kStepMinChunkRows ? cap : kStepMinChunkRows;
+  return rc >= need ? rc : 0;
 }
 }  // namespace
 
@@ -517,17 +626,19 @@ size_t a3po_train_step_min_workspace_bytes(int64_t N, int H, int V, a3po_dtype d
 
 size_t a3po_train_step_workspace_bytes(int64_t N, int H, int V, a3po_dtype dt) {
   if (N < 0 || H <= 0 || V <= 0) return 0;
-  size_t a = a3po_token_logprobs_workspace_bytes(N, H, V, dt, 0);
-  const size_t b = a3po_token_logprobs_workspace_bytes(N, H, V, dt, 1);
-  const size_t c = a3po_loss_workspace_bytes(N);
-  if (b > a) a = b;
-  if (c > a) a = c;
-  if (dt == A3PO_BF16 && N > 0) {
-    // Keeping the logits costs N x V x 4 bytes of workspace (kept logits + dz, both for all N rows since the
-    // number of rows that take part is only known on the device).  It is recommended up to 96 GiB; beyond that
-    // the recommendation is the recomputing path's size (a caller may still pass more).
-    const size_t d = saved_step_layout(N, H, V).total;
-    if (d > a && d <= (static_cast<size_t>(96) << 30)) a = d;
+  size_t a = a3po_train_step_min_workspace_bytes(N, H, V, dt);
+  if (dt == A3PO_BF16 && N > 0 && H % 8 == 0) {
+    // the keeping path: kept ratios for one chunk of up to kStepChunkRows rows (about 2 V bytes per row) plus
+    // buffers that scale with N x H; a caller may pass more and gets larger chunks (fewer launches)
+    long long rc = compact_capacity(N);
+    if (rc > kStepChunkRows) rc = kStepChunkRows;
+    const size_t d = step_layout(N, H, V, rc).total;
+    if (d > a) a = d;
+  } else {
+    size_t f = a3po_token_logprobs_workspace_bytes(N, H, V, dt, 0);
+    const size_t b = a3po_token_logprobs_workspace_bytes(N, H, V, dt, 1);
+    if (b > f) f = b;
+    if (f > a) a = f;
   }
   return a;
 }
@@ -535,19 +646,21 @@ size_t a3po_train_step_workspace_bytes(int64_t N, int H, int V, a3po_dtype dt) {
 int a3po_train_step(const void* hidden, const int32_t* targets, const float* behav_logp, const int32_t* versions,
                     const float* adv, const uint8_t* mask, int64_t N, int H, int V, a3po_dtype dt,
                     int32_t current_version, float clip_eps, float inv_temperature, const void* w, float* grad_w,
-                    int accumulate_grad_w, void* grad_hidden, float* logp, float* lse, float* grad_logp, float* loss,
-                    a3po_stats* stats, void* ws, size_t ws_bytes, uint32_t* status, void* stream_) {
+                    int accumulate_grad_w, void* grad_hidden, float* logp, float* lse, float* entropy,
+                    float* grad_logp, float* loss, a3po_stats* stats, void* ws, size_t ws_bytes, uint32_t* status,
+                    void* stream_) {
   A3PO_RETURN_IF(check_lmhead_args(hidden, w, targets, N, H, V, dt, inv_temperature));
-  if (!grad_w || !loss || (N > 0 && (!behav_logp || !versions || !adv || !mask || !grad_hidden || !logp || !lse ||
-                                      !grad_logp)))
+  if (!grad_w || !loss || !(clip_eps >= 0.f) ||
+      (N > 0 && (!behav_logp || !versions || !adv || !mask || !grad_hidden || !logp || !lse || !grad_logp)))
     return A3PO_ERR_INVALID_ARG;
   if (!ws || !aligned_to(ws, 256)) return A3PO_ERR_WORKSPACE;
-  const bool keep_logits = N > 0 && use_tc(dt, hidden, w, N, H, V) && !env_flag("A3PO_NO_SAVED_LOGITS") &&
-                           ws_bytes >= saved_step_layout(N, H, V).total && aligned_to(grad_hidden, 16) &&
-                           aligned_to(grad_w, 16);
-  if (!keep_logits) {
+  const long long chunk_rows = (N > 0 && use_tc(dt, hidden, w, N, H, V) && aligned_to(grad_hidden, 16) &&
+                                aligned_to(grad_w, 16))
+                                   ? step_chunk_rows_for(ws_bytes, N, H, V)
+                                   : 0;
+  if (chunk_rows == 0) {
     // three independent calls; the backward recomputes the logits chunk by chunk
-    A3PO_RETURN_IF(a3po_token_logprobs_fwd(hidden, w, targets, mask, N, H, V, dt, inv_temperature, logp, lse, nullptr,
+    A3PO_RETURN_IF(a3po_token_logprobs_fwd(hidden, w, targets, mask, N, H, V, dt, inv_temperature, logp, lse, entropy,
                                            ws, ws_bytes, status, stream_));
     A3PO_RETURN_IF(a3po_loss_fwd_bwd(logp, behav_logp, versions, 0, nullptr, 0, current_version, adv, mask, N,
                                      clip_eps, 1, loss, stats, grad_logp, ws, ws_bytes, stream_));
@@ -555,17 +668,72 @@ int a3po_train_step(const void* hidden, const int32_t* targets, const float* beh
                                    grad_w, accumulate_grad_w, ws, ws_bytes, status, stream_);
   }
 
-  // ---- forward keeping its logits (rows with mask != 0), loss on every token, backward from the kept logits
-  const SavedStepLayout lay = saved_step_layout(N, H, V);
+  // ---- rows with mask != 0 are gathered once; then, per chunk of those rows: forward keeping the softmax ->
+  // loss forward + backward (M is the number of gathered rows, known up front) -> the two gradient contractions
+  cudaStream_t stream = as_stream(stream_);
+  const StepLayout lay = step_layout(N, H, V, chunk_rows);
+  if (lay.total > ws_bytes) return A3PO_ERR_WORKSPACE;
   char* base = static_cast<char*>(ws);
-  A3PO_RETURN_IF(a3po_token_logprobs_fwd_keep(hidden, w, targets, mask, N, H, V, inv_temperature, logp, lse,
-                                              base + lay.kept, lay.kept_bytes, base + lay.call_ws, lay.call_ws_bytes,
-                                              status, stream_));
-  A3PO_RETURN_IF(a3po_loss_fwd_bwd(logp, behav_logp, versions, 0, nullptr, 0, current_version, adv, mask, N, clip_eps,
-                                   1, loss, stats, grad_logp, base + lay.loss, a3po_loss_workspace_bytes(N), stream_));
-  return a3po_token_logprobs_bwd_kept(hidden, w, targets, lse, grad_logp, base + lay.kept, lay.kept_bytes, N, H, V,
-                                      inv_temperature, grad_hidden, grad_w, accumulate_grad_w, base + lay.call_ws,
-                                      lay.call_ws_bytes, status, stream_);
+  const long long cap = compact_capacity(N);
+  CompactBuffers cb;
+  cb.cap = cap;
+  cb.count = reinterpret_cast<int*>(base + lay.count);
+  cb.block_counts = reinterpret_cast<int*>(base + lay.scan);
+  cb.block_offsets = cb.block_counts + 4096;
+  cb.pos = reinterpret_cast<int*>(base + lay.pos);
+  cb.idx = reinterpret_cast<int*>(base + lay.idx);
+  cb.targets_c = reinterpret_cast<int32_t*>(base + lay.targets_c);
+  cb.hidden_c = reinterpret_cast<__nv_bfloat16*>(base + lay.hidden_c);
+  cb.lse_c = nullptr;
+  cb.g_c = nullptr;
+  cb.grad_hidden_c = nullptr;
+  auto f32 = [&](size_t off) { return reinterpret_cast<float*>(base + off); };
+  float *zy = f32(lay.zy), *sprime = f32(lay.sprime), *logp_c = f32(lay.logp_c), *lse_c = f32(lay.lse_c);
+  float *g_c = f32(lay.g_c), *ent_c = f32(lay.ent_c), *behav_c = f32(lay.behav_c), *adv_c = f32(lay.adv_c);
+  float* row_scale = f32(lay.row_scale);
+  int32_t* versions_c = reinterpret_cast<int32_t*>(base + lay.versions_c);
+  uint8_t* mask_c = reinterpret_cast<uint8_t*>(base + lay.mask_c);
+  long long* n_valid = reinterpret_cast<long long*>(base + lay.n_valid);
+  char* partials = base + lay.partials;
+  float *part_s = f32(lay.part_s), *part_e = f32(lay.part_e);
+  void* q = base + lay.q;
+  __nv_bfloat16* hs = reinterpret_cast<__nv_bfloat16*>(base + lay.hs);
+  __nv_bfloat16* ghc = reinterpret_cast<__nv_bfloat16*>(base + lay.ghc);
+  const __nv_bfloat16* hidden_c = cb.hidden_c;
+
+  const int n_chunks = static_cast<int>((cap + chunk_rows - 1) / chunk_rows);
+  int max_blocks = loss_max_partials() / n_chunks;
+  if (max_blocks < 1) return A3PO_ERR_WORKSPACE;   // more than 4096 chunks: the workspace is far too small for N
+  const int loss_blocks = loss_blocks_for(chunk_rows, max_blocks);
+
+  A3PO_RETURN_IF(compact_rows(hidden, H, targets, mask, nullptr, nullptr, N, cb, stream));
+  A3PO_RETURN_IF(gather_loss_inputs(cb.idx, cb.count, cap, behav_logp, versions, adv, behav_c, versions_c, adv_c,
+                                    mask_c, n_valid, stream));
+  A3PO_RETURN_IF(flag_bad_targets(targets, N, V, status, stream));
+  for (int i = 0; i < n_chunks; ++i) {
+    const long long c0 = static_cast<long long>(i) * chunk_rows;
+    const long long rows = (c0 + chunk_rows <= cap) ? chunk_rows : cap - c0;
+    const int splits = lmhead_tc_fwd_splits(rows, V);
+    A3PO_RETURN_IF(target_logits(hidden_c, w, cb.targets_c, cb.count, c0, rows, H, V, inv_temperature, zy, stream));
+    A3PO_RETURN_IF(lmhead_fwd_keep_tc(hidden_c + c0 * H, w, cb.targets_c + c0, zy + c0, rows, H, V, inv_temperature,
+                                      splits, part_s, entropy ? part_e : nullptr, q, cb.count, c0, status, stream));
+    A3PO_RETURN_IF(merge_kept(part_s, part_e, zy, cb.count, c0, rows, splits, inv_temperature, sprime, logp_c, lse_c,
+                              entropy ? ent_c : nullptr, status, stream));
+    A3PO_RETURN_IF(loss_fwd_bwd_slice(logp_c + c0, behav_c + c0, versions_c + c0, adv_c + c0, mask_c + c0, rows,
+                                      current_version, clip_eps, n_valid, g_c + c0,
+                                      partials + static_cast<size_t>(i) * loss_blocks * loss_partial_bytes(),
+                                      loss_blocks, stream));
+    A3PO_RETURN_IF(prepare_kept_backward(cb.count, c0, rows, H, V, inv_temperature, sprime, cb.targets_c, g_c, nullptr,
+                                         cb.idx, hidden_c, nullptr, row_scale, q, hs, stream));
+    A3PO_RETURN_IF(lmhead_grad_hidden_from_kept_tc(q, w, row_scale + c0, rows, H, V, ghc, cb.count, c0, status,
+                                                   stream));
+    A3PO_RETURN_IF(scatter_rows_range(ghc, H, cb.idx, cb.count, c0, rows, grad_hidden, stream));
+    A3PO_RETURN_IF(lmhead_grad_w_from_kept_tc(q, hs, rows, H, V, grad_w, (accumulate_grad_w || i > 0) ? 1 : 0,
+                                              (i == 0 && !accumulate_grad_w) ? 1 : 0, cb.count, c0, status, stream));
+  }
+  A3PO_RETURN_IF(finish_batch_outputs(cb.pos, N, logp_c, logp, lse_c, lse, g_c, grad_logp, ent_c, entropy,
+                                      grad_hidden, H, stream));
+  return loss_finalize_partials(partials, n_chunks * loss_blocks, loss, stats, stream);
 }
 
 int a3po_train_step_host(const void* h_hidden, const int32_t* h_targets, const float* h_behav_logp,
@@ -588,11 +756,14 @@ int a3po_train_step_host(const void* h_hidden, const int32_t* h_targets, const f
   auto h2d = [&](size_t off, const void* src, size_t bytes) -> bool {
     return bytes == 0 || cudaMemcpyAsync(base + off, src, bytes, cudaMemcpyHostToDevice, stream) == cudaSuccess;
   };
-  if (!h2d(s.hidden, h_hidden, rows * H * elt_size(dt)) || !h2d(s.targets, h_targets, rows * 4) ||
-      !h2d(s.behav, h_behav_logp, rows * 4) || !h2d(s.versions, h_versions, rows * 4) ||
-      !h2d(s.adv, h_adv, rows * 4) || !h2d(s.mask, h_mask, rows)) {
-    cudaGetLastError();
-    return A3PO_ERR_CUDA;
+  {
+    ProfileScope scope(kKH2D, stream);   // with the per-kernel profile on, the copies show up as one entry
+    if (!h2d(s.hidden, h_hidden, rows * H * elt_size(dt)) || !h2d(s.targets, h_targets, rows * 4) ||
+        !h2d(s.behav, h_behav_logp, rows * 4) || !h2d(s.versions, h_versions, rows * 4) ||
+        !h2d(s.adv, h_adv, rows * 4) || !h2d(s.mask, h_mask, rows)) {
+      cudaGetLastError();
+      return A3PO_ERR_CUDA;
+    }
   }
   const void* hidden = base + s.hidden;
   const int32_t* targets = reinterpret_cast<const int32_t*>(base + s.targets);
@@ -607,7 +778,7 @@ int a3po_train_step_host(const void* h_hidden, const int32_t* h_targets, const f
   a3po_stats* stats = reinterpret_cast<a3po_stats*>(base + s.stats);
 
   A3PO_RETURN_IF(a3po_train_step(hidden, targets, behav, versions, adv, mask, N, H, V, dt, current_version, clip_eps,
-                                 inv_temperature, d_w, d_grad_w, accumulate_grad_w, d_grad_hidden, logp, lse,
+                                 inv_temperature, d_w, d_grad_w, accumulate_grad_w, d_grad_hidden, logp, lse, nullptr,
                                  grad_logp, loss, stats, d_ws, ws_bytes, d_status, stream_));
   if (cudaMemcpyAsync(h_loss, loss, sizeof(float), cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
       (h_stats && cudaMemcpyAsync(h_stats, stats, sizeof(a3po_stats), cudaMemcpyDeviceToHost, stream) != cudaSuccess)) {

@@ -62,20 +62,64 @@ int lmhead_bwd_tc(const void* hidden, const void* w, const int32_t* targets, con
                   int accumulate, void* ws, size_t ws_bytes, long long chunk_rows, const int* dyn_rows,
                   uint32_t* status, cudaStream_t stream);
 
-// ---- backward without recomputation (lmhead_tc.cu, saved_logits.cu) ----
-// The saving forward keeps, for n rows, u[n, v^8] (fp16: z log2(e)/T minus a per-(row, 256-column tile)
-// reference) followed by ref[n, tiles] (fp32) in one buffer of lmhead_tc_saved_logits_bytes(n, v) bytes.
-size_t lmhead_tc_saved_logits_bytes(long long n, int v);
-int lmhead_fwd_save_tc(const void* hidden, const void* w, const int32_t* targets, long long n, int h, int v,
-                       float inv_t, int splits, SoftmaxPartial* part, float* zy, void* saved, const int* dyn_rows,
-                       uint32_t* status, cudaStream_t stream);
-// dz[c, :] (bf16, pitch v^8, `bwd.cap` rows allocated) for the backward's compact rows from the kept logits;
-// fwd_pos maps a batch row to its row in `saved` (null: identity).
-int dz_from_saved(const void* saved, long long saved_rows, int v, const int* fwd_pos, const CompactBuffers& bwd,
-                  float inv_t, void* dz, cudaStream_t stream);
-int lmhead_bwd_from_dz_tc(const void* hidden, const void* w, const void* dz, long long n, int h, int v,
-                          void* grad_hidden, float* grad_w, int accumulate, const int* dyn_rows, uint32_t* status,
-                          cudaStream_t stream);
+// ---- backward without recomputation (lmhead_tc.cu, kept_rows.cu) ----
+// The keeping forward works on rows [offset, offset + n) of a compact row space whose size is *dyn_rows and leaves,
+// for each row, q[r, v] = exp(z[r, v] - zy[r]) in bf16 (pitch v^8, 0 at the target column) and per-split sums of q
+// (the target left out).  zy is the row's target logit / T, computed beforehand by target_logits().
+size_t lmhead_tc_kept_bytes(long long rows, int v);
+int lmhead_fwd_keep_tc(const void* hidden, const void* w, const int32_t* targets, const float* zy, long long n, int h,
+                       int v, float inv_t, int splits, float* part_s, float* part_e, void* q, const int* dyn_rows,
+                       long long dyn_offset, uint32_t* status, cudaStream_t stream);
+int lmhead_grad_hidden_from_kept_tc(const void* q, const void* w, const float* row_scale, long long n, int h, int v,
+                                    void* grad_hidden, const int* dyn_rows, long long dyn_offset, uint32_t* status,
+                                    cudaStream_t stream);
+int lmhead_grad_w_from_kept_tc(const void* q, const void* hs, long long n, int h, int v, float* grad_w, int accumulate,
+                               int zero_when_empty, const int* dyn_rows, long long dyn_offset, uint32_t* status,
+                               cudaStream_t stream);
+
+// Small per-row kernels around the kept-ratio path (kept_rows.cu).  `count` is the device-resident size of the
+// compact row space; every launch covers compact rows [offset, offset + rows) and arrays are indexed by compact row
+// unless they say otherwise.
+// zy[c] = dot(hidden_c[c, :], W[targets_c[c], :]) / T for the rows a GEMM launch may touch (up to the next 128).
+int target_logits(const void* hidden_c, const void* w, const int32_t* targets_c, const int* count, long long offset,
+                  long long rows, int h, int v, float inv_t, float* zy, cudaStream_t stream);
+// s = sum of the split sums; lse = zy + log1p(s), logp = -log1p(s), sprime = s,
+// entropy = lse - (zy + part_e / T) / (1 + s); rows at and beyond *count get zeros.  part_* are [splits][rows].
+int merge_kept(const float* part_s, const float* part_e, const float* zy, const int* count, long long offset,
+               long long rows, int splits, float inv_t, float* sprime, float* logp, float* lse, float* entropy,
+               uint32_t* status, cudaStream_t stream);
+// Per-token inputs of the loss in the compact row space (rows beyond *count: zeros, mask 0), and *n_valid = *count.
+int gather_loss_inputs(const int* idx, const int* count, long long cap, const float* behav, const int32_t* versions,
+                       const float* adv, float* behav_c, int32_t* versions_c, float* adv_c, uint8_t* mask_c,
+                       long long* n_valid, cudaStream_t stream);
+// Prepares the two gradient contractions for rows [offset, offset + rows):
+//   row_scale[c] = -g / (T (1 + sprime[c]))     g = g_c[c], or g_batch[idx[c]] when g_c is null
+//   q[c - offset, y_c] = -sprime[c]              (the target's entry: 1 - 1/p_y)
+//   hs[c - offset, :]  = row_scale[c] * hidden row   (hidden_c[c], or hidden_batch[idx[c]] when hidden_c is null)
+// rows from *count to the next multiple of 128 get scale 0 and zero hs rows.
+int prepare_kept_backward(const int* count, long long offset, long long rows, int h, int v, float inv_t,
+                          const float* sprime, const int32_t* targets_c, const float* g_c, const float* g_batch,
+                          const int* idx, const void* hidden_c, const void* hidden_batch, float* row_scale, void* q,
+                          void* hs, cudaStream_t stream);
+// dst[idx[c], :] = src[c - offset, :] for compact rows c in [offset, min(offset + rows, *count)).
+int scatter_rows_range(const void* src, int h, const int* idx, const int* count, long long offset, long long rows,
+                       void* dst, cudaStream_t stream);
+// Batch-space outputs from compact ones: out[t] = pos[t] >= 0 ? in_c[pos[t]] : 0 for up to four arrays (null = skip),
+// and, when grad_hidden is given, zero rows of grad_hidden [n, h] for rows that were not kept.
+int finish_batch_outputs(const int* pos, long long n, const float* logp_c, float* logp, const float* lse_c, float* lse,
+                         const float* g_c, float* grad_logp, const float* ent_c, float* entropy, void* grad_hidden,
+                         int h, cudaStream_t stream);
+
+// ---- loss on a slice, for the row-chunked step (loss_kernels.cu) ----
+// Forward + backward of the A-3PO loss on n tokens with M taken from *n_valid; block partials go to
+// partials[0 .. blocks) (loss_partial_bytes() each), which loss_finalize_partials sums in index order.
+size_t loss_partial_bytes();
+int loss_max_partials();
+int loss_blocks_for(long long n, int max_blocks);
+int loss_fwd_bwd_slice(const float* logp, const float* behav, const int32_t* versions, const float* adv,
+                       const uint8_t* mask, long long n, int32_t current_version, float clip_eps,
+                       const long long* n_valid, float* grad_logp, void* partials, int blocks, cudaStream_t stream);
+int loss_finalize_partials(const void* partials, int count, float* loss, a3po_stats* stats, cudaStream_t stream);
 
 // Launches a one-warp kernel whose bounded wait must expire after timeout_ms and set the status bit.
 int selftest_wait_timeout(uint32_t* status, unsigned timeout_ms, cudaStream_t stream);

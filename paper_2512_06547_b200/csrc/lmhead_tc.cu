@@ -4,17 +4,20 @@
 //     C[M, N] = A[M, K] * B[N, K]^T,
 // and differs only in its epilogue:
 //   forward      A = hidden, B = W           online (max, sum-exp) per row + target gather
-//   forward+keep same, and the shifted logits are kept in fp16 for a backward without recomputation
+//   forward+keep same, and every probability is kept as a bf16 ratio to the target token's for a backward
+//                without recomputation
 //   dz           A = hidden, B = W           dz = g (1[v = y] - exp(z - lse)) -> bf16 chunk of rows
-//   grad_hidden  A = dz,     B = W^T         bf16 store            (W read in place as an N-major operand)
+//   grad_hidden  A = dz,     B = W^T         bf16 store, optional per-row scale (W read in place, N-major)
 //   grad_w       A = dz^T,   B = hidden^T    fp32 store/accumulate (both read in place, M-/N-major)
+// (with kept probability ratios in place of dz the per-row factor of dz moves into the grad_hidden epilogue
+// and into the hidden operand of grad_w)
 //
 // Per CTA (one per SM): warp 0 = TMA producer (one elected lane), warp 1 = tcgen05.mma issuer
 // (one elected lane; it also owns the TMEM allocation), warps 2-5 = epilogue (one TMEM lane
 // quarter each, one accumulator row per thread).  Operand tiles (128 x 64 and 256 x 64 bf16,
 // 128-byte swizzle) move through a 4-stage shared-memory ring guarded by full/empty mbarriers;
 // the 128 x 256 fp32 accumulator is double-buffered in TMEM (2 x 256 columns) so the epilogue
-// of tile i overlaps the MMAs of tile i+1.  Output tiles (kept logits, dz, gradients) leave through
+// of tile i overlaps the MMAs of tile i+1.  Output tiles (kept ratios, dz, gradients) leave through
 // two swizzled shared-memory slabs and TMA tile stores.  The full logits matrix never exists: the
 // plain forward keeps nothing, the keeping forward writes only the rows that take part, into scratch.
 //
@@ -166,7 +169,6 @@ struct SlabStore;  // output staging for TMA stores, defined below
 template <bool ENT>
 struct FwdEpilogue {
   static constexpr int kKernelId = kKTcFwd;
-  static constexpr bool kTwoPass = false;
   struct Params {
     const int32_t* targets;
     long long n;
@@ -277,7 +279,6 @@ struct SlabStore {
 
 struct DzEpilogue {
   static constexpr int kKernelId = kKTcDz;
-  static constexpr bool kTwoPass = false;
   struct Params {
     const int32_t* targets;   // indexed by global token row
     const float* lse;
@@ -334,130 +335,105 @@ struct DzEpilogue {
   __device__ __forceinline__ void end(const Params&, long long, int) {}
 };
 
-__device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
-  __half2 p = __floats2half2_rn(lo, hi);
-  return *reinterpret_cast<uint32_t*>(&p);
-}
-
-// Forward that also keeps the logits for the backward, so that the backward need not recompute
-// them: u[row, v] = z[row, v] * log2(e) / T - ref[row, tile] in fp16 and ref[row, tile] in fp32,
-// where ref is the row's running maximum when the 256-column tile starts (u is then near or below
-// zero, so the entries that matter for the softmax are the accurately stored ones).  The first tile
-// of a work item has no running maximum yet: it is swept twice in TMEM, first for its row maxima,
-// then for the exponentials and the stores.
-struct FwdSaveEpilogue {
-  static constexpr int kKernelId = kKTcFwdSave;
-  static constexpr bool kTwoPass = true;
+// Forward that also keeps the row's softmax for the backward, so that the backward need not recompute
+// the logits.  The reference of row t is its own target logit zy (computed beforehand, one dot product
+// per row), and what is kept is the probability ratio
+//     q[t, v] = exp(z[t, v] - zy[t]) = p[t, v] / p[t, y_t]                  (bf16, 0 at v = y_t)
+// A ratio is a floating-point number with bf16's uniform relative precision whatever its size, so
+// peaked and flat rows are kept equally well, and every split of a row shares the one reference, so
+// no running maximum, rescaling or extra sweep is needed.  The target column is left out of the sum:
+//     s[t] = sum_{v != y_t} q[t, v],  lse = zy + log1p(s),  logp = -log1p(s),  1 - p_y = s / (1 + s),
+// which stays accurate when p_y approaches 1.  The exponent is clamped at 126 (a ratio above 2^126
+// means p_y < 1e-37; the merge flags such a row).
+template <bool ENT>
+struct KeepEpilogue {
+  static constexpr int kKernelId = kKTcFwdKeep;
   struct Params {
-    const int32_t* targets;
+    const int32_t* targets;   // [n] rows of this launch
+    const float* zy;          // [n] target logit / T, natural-log units
     long long n;
     int v;
-    int vpad;      // row pitch of u
-    int n_tiles;   // row pitch of ref
+    int vpad;                 // row pitch of q
     float scale_log2;
     float inv_t;
-    SoftmaxPartial* part;
-    float* zy;
-    __half* u;     // [n, vpad]
-    float* ref;    // [n, n_tiles]
+    float* part_s;            // [splits][n] sum of the ratios over the split's columns, target left out
+    float* part_e;            // [splits][n] sum of ratio * raw logit (entropy), or null
+    __nv_bfloat16* q;         // [n, vpad]
   };
-  static int make_c_map(const Params& p, CUtensorMap* map) {
-    return make_out_map(map, p.u, 2, p.v, p.n, p.vpad);  // 2-byte elements: a plain copy, the type does not matter
-  }
-  float m, s, tmax, ref_tile;
+  static int make_c_map(const Params& p, CUtensorMap* map) { return make_out_map(map, p.q, 2, p.v, p.n, p.vpad); }
+  float s, e, ref2;
   int y;
-  long long row;
   uint8_t* cur;
-  __device__ __forceinline__ void begin(const Params& p, long long row_) {
-    row = row_;
-    m = -INFINITY; s = 0.f;
+  __device__ __forceinline__ void begin(const Params& p, long long row) {
+    s = 0.f; e = 0.f; ref2 = 0.f;
     y = -1;
-    if (row < p.n) y = min(max(p.targets[row], 0), p.v - 1);
-  }
-  __device__ __forceinline__ void tile_begin() { tmax = -INFINITY; }
-  __device__ __forceinline__ void prepass(const Params& p, int col0, uint32_t (&r)[kEpiChunk]) {
-    if (col0 + kEpiChunk > p.v) {
-#pragma unroll
-      for (int j = 0; j < kEpiChunk; ++j)
-        if (col0 + j >= p.v) r[j] = 0xff800000u;  // -inf: columns past V do not exist
+    if (row < p.n) {
+      y = min(max(p.targets[row], 0), p.v - 1);
+      ref2 = p.zy[row] * kLog2e;
     }
-#pragma unroll
-    for (int j = 0; j < kEpiChunk; ++j) tmax = fmaxf(tmax, bits_to_float(r[j]));
-  }
-  // Fixes the tile's reference: the running maximum at this point (after the extra sweep for an
-  // item's first tile).  Later columns of the tile may exceed it, which only makes u slightly positive.
-  __device__ __forceinline__ void tile_ready(const Params& p, int tile) {
-    const float xm = tmax * p.scale_log2;  // -inf unless the extra sweep ran
-    if (xm > m) {
-      s *= fast_exp2(m - xm);
-      m = xm;
-    }
-    ref_tile = m;
-    if (row < p.n) p.ref[row * p.n_tiles + tile] = ref_tile;
   }
   __device__ __forceinline__ void chunk(const Params& p, int tile_row0, int col0, uint32_t (&r)[kEpiChunk],
                                         SlabStore& st) {
     if (col0 + kEpiChunk > p.v) {
 #pragma unroll
       for (int j = 0; j < kEpiChunk; ++j)
-        if (col0 + j >= p.v) r[j] = 0xff800000u;
+        if (col0 + j >= p.v) r[j] = 0xff800000u;  // -inf: columns past V do not exist
     }
-    float zmax = -INFINITY;
+    float q[kEpiChunk];
 #pragma unroll
-    for (int j = 0; j < kEpiChunk; ++j) zmax = fmaxf(zmax, bits_to_float(r[j]));
-    const float xm = zmax * p.scale_log2;
-    if (xm > m) {
-      s *= fast_exp2(m - xm);
-      m = xm;
-    }
-    const float back = ref_tile - m;  // <= 0: from the tile's reference to the running maximum
-    float x[kEpiChunk];
-    float acc = 0.f;
-#pragma unroll
-    for (int j = 0; j < kEpiChunk; ++j) {
-      x[j] = fmaf(bits_to_float(r[j]), p.scale_log2, -ref_tile);
-      acc += fast_exp2(x[j] + back);
-    }
-    s += acc;
+    for (int j = 0; j < kEpiChunk; ++j)
+      q[j] = fast_exp2(fminf(fmaf(bits_to_float(r[j]), p.scale_log2, -ref2), 126.f));
     if (y >= col0 && y < col0 + kEpiChunk) {
-      float zyv = 0.f;
 #pragma unroll
       for (int j = 0; j < kEpiChunk; ++j)
-        if (col0 + j == y) zyv = bits_to_float(r[j]);
-      p.zy[row] = zyv * p.inv_t;
+        if (col0 + j == y) q[j] = 0.f;   // the target's own entry is written by the backward (-s)
     }
+    float acc = 0.f, ee = 0.f;
+#pragma unroll
+    for (int j = 0; j < kEpiChunk; ++j) {
+      acc += q[j];
+      if (ENT) ee = fmaf(q[j], q[j] > 0.f ? bits_to_float(r[j]) : 0.f, ee);
+    }
+    s += acc;
+    if (ENT) e += ee;
     const int half = (col0 >> 5) & 1;
     if (half == 0) cur = st.acquire();
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
+    for (int k = 0; k < 4; ++k) {
       uint4 w;
-      w.x = pack_half2(x[q * 8 + 0], x[q * 8 + 1]);
-      w.y = pack_half2(x[q * 8 + 2], x[q * 8 + 3]);
-      w.z = pack_half2(x[q * 8 + 4], x[q * 8 + 5]);
-      w.w = pack_half2(x[q * 8 + 6], x[q * 8 + 7]);
-      *st.piece(cur, half * 4 + q) = w;
+      w.x = pack_bf16x2(q[k * 8 + 0], q[k * 8 + 1]);
+      w.y = pack_bf16x2(q[k * 8 + 2], q[k * 8 + 3]);
+      w.z = pack_bf16x2(q[k * 8 + 4], q[k * 8 + 5]);
+      w.w = pack_bf16x2(q[k * 8 + 6], q[k * 8 + 7]);
+      *st.piece(cur, half * 4 + k) = w;
     }
     if (half == 1) st.submit(cur, col0 - 32, tile_row0, col0 - 32 < p.v, false);
   }
-  __device__ __forceinline__ void end(const Params& p, long long row_, int split) {
-    if (row_ < p.n) p.part[static_cast<long long>(split) * p.n + row_] = SoftmaxPartial{m * kLn2, s};
+  __device__ __forceinline__ void end(const Params& p, long long row, int split) {
+    if (row < p.n) {
+      p.part_s[static_cast<long long>(split) * p.n + row] = s;
+      if (ENT) p.part_e[static_cast<long long>(split) * p.n + row] = e;
+    }
   }
 };
 
 struct StoreBf16Epilogue {
   static constexpr int kKernelId = kKTcGradHidden;
-  static constexpr bool kTwoPass = false;
   struct Params {
     __nv_bfloat16* c;
     long long ldc;
     long long m_rows;
     int n_cols;  // multiple of 8
+    const float* row_scale;  // [m_rows] factor applied to each output row, or null for none
   };
   static int make_c_map(const Params& p, CUtensorMap* map) {
     return make_out_map(map, p.c, 2, p.n_cols, p.m_rows, p.ldc);
   }
   uint8_t* cur;
-  __device__ __forceinline__ void begin(const Params&, long long) {}
+  float sc;
+  __device__ __forceinline__ void begin(const Params& p, long long row) {
+    sc = (p.row_scale != nullptr && row < p.m_rows) ? p.row_scale[row] : 1.0f;
+  }
   __device__ __forceinline__ void chunk(const Params& p, int tile_row0, int col0, uint32_t (&r)[kEpiChunk],
                                         SlabStore& st) {
     const int half = (col0 >> 5) & 1;
@@ -465,10 +441,10 @@ struct StoreBf16Epilogue {
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
       uint4 u;
-      u.x = pack_bf16x2(bits_to_float(r[q * 8 + 0]), bits_to_float(r[q * 8 + 1]));
-      u.y = pack_bf16x2(bits_to_float(r[q * 8 + 2]), bits_to_float(r[q * 8 + 3]));
-      u.z = pack_bf16x2(bits_to_float(r[q * 8 + 4]), bits_to_float(r[q * 8 + 5]));
-      u.w = pack_bf16x2(bits_to_float(r[q * 8 + 6]), bits_to_float(r[q * 8 + 7]));
+      u.x = pack_bf16x2(sc * bits_to_float(r[q * 8 + 0]), sc * bits_to_float(r[q * 8 + 1]));
+      u.y = pack_bf16x2(sc * bits_to_float(r[q * 8 + 2]), sc * bits_to_float(r[q * 8 + 3]));
+      u.z = pack_bf16x2(sc * bits_to_float(r[q * 8 + 4]), sc * bits_to_float(r[q * 8 + 5]));
+      u.w = pack_bf16x2(sc * bits_to_float(r[q * 8 + 6]), sc * bits_to_float(r[q * 8 + 7]));
       *st.piece(cur, half * 4 + q) = u;
     }
     if (half == 1) st.submit(cur, col0 - 32, tile_row0, col0 - 32 < p.n_cols, false);
@@ -478,7 +454,6 @@ struct StoreBf16Epilogue {
 
 struct StoreF32Epilogue {
   static constexpr int kKernelId = kKTcGradW;
-  static constexpr bool kTwoPass = false;
   struct Params {
     float* c;
     long long ldc;
@@ -679,21 +654,6 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           tcgen05_fence_after_sync();
         }
         const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(acc * BN);
-        if constexpr (Epi::kTwoPass) {
-          // an extra sweep over the first accumulator tile of an item: the epilogue learns the row maxima it
-          // uses as the first reference (later tiles take the running maximum they start with)
-          epi.tile_begin();
-          if (nt == it.n_begin) {
-#pragma unroll 1
-            for (int c = 0; c < BN / kEpiChunk; ++c) {
-              uint32_t r[kEpiChunk];
-              tmem_ld_32x32(taddr + static_cast<uint32_t>(c * kEpiChunk), r);
-              tmem_ld_wait();
-              epi.prepass(ep, nt * BN + c * kEpiChunk, r);
-            }
-          }
-          epi.tile_ready(ep, nt);
-        }
 #pragma unroll 1
         for (int c = 0; c < BN / kEpiChunk; ++c) {
           uint32_t r[kEpiChunk];
@@ -757,13 +717,18 @@ int make_map(CUtensorMap* map, const Operand& op, bool mn_major, int tile_mn) {
   return r == CUDA_SUCCESS ? A3PO_OK : A3PO_ERR_CUDA;
 }
 
-// C[M, N] = sum_k A[m, k] B[n, k];  splits = 0 means one column tile per work item.
-// Tuning overrides read from the environment (positive integers); used for sweeps, not needed in normal use.
+// Tuning overrides (positive integers read from the environment) exist only in builds made with
+// -DA3PO_TUNING, for sweeps; a normal build takes the defaults and reads no environment variable.
 int tuning_override(const char* name, int fallback) {
+#ifdef A3PO_TUNING
   const char* e = std::getenv(name);
   if (!e) return fallback;
   const int v = std::atoi(e);
   return v > 0 ? v : fallback;
+#else
+  (void)name;
+  return fallback;
+#endif
 }
 
 // Device-resident row count for a launch (see ItemMap).
@@ -775,6 +740,7 @@ struct DynRows {
   long long cap = 0;
 };
 
+// C[M, N] = sum_k A[m, k] B[n, k];  splits = 0 means one column tile per work item.
 template <class Epi, bool A_MN, bool B_MN>
 int launch_gemm(const Operand& a, const Operand& b, int splits, const typename Epi::Params& ep, const DynRows& dyn,
                 uint32_t* status, cudaStream_t stream) {
@@ -868,26 +834,29 @@ int lmhead_fwd_tc(const void* hidden, const void* w, const int32_t* targets, lon
   return launch_gemm<FwdEpilogue<false>, false, false>(a, b, splits, p, dyn, status, stream);
 }
 
-size_t lmhead_tc_saved_logits_bytes(long long n, int v) {
+size_t lmhead_tc_kept_bytes(long long rows, int v) {
   const size_t vpad = round_up(static_cast<size_t>(v), 8);
-  const size_t n_tiles = static_cast<size_t>((v + BN - 1) / BN);
-  return round_up(static_cast<size_t>(n) * vpad * 2, 256) + round_up(static_cast<size_t>(n) * n_tiles * 4, 256);
+  return round_up(static_cast<size_t>(rows > 0 ? rows : 0) * vpad * 2, 256);
 }
 
-int lmhead_fwd_save_tc(const void* hidden, const void* w, const int32_t* targets, long long n, int h, int v,
-                       float inv_t, int splits, SoftmaxPartial* part, float* zy, void* saved, const int* dyn_rows,
-                       uint32_t* status, cudaStream_t stream) {
+int lmhead_fwd_keep_tc(const void* hidden, const void* w, const int32_t* targets, const float* zy, long long n, int h,
+                       int v, float inv_t, int splits, float* part_s, float* part_e, void* q, const int* dyn_rows,
+                       long long dyn_offset, uint32_t* status, cudaStream_t stream) {
   const Operand a{hidden, n, h, h};
   const Operand b{w, v, h, h};
   DynRows dyn;
   dyn.rows = dyn_rows;
+  dyn.offset = dyn_offset;
   dyn.cap = n;
   const int vpad = static_cast<int>(round_up(static_cast<size_t>(v), 8));
-  const int n_tiles = (v + BN - 1) / BN;
-  __half* u = static_cast<__half*>(saved);
-  float* ref = reinterpret_cast<float*>(static_cast<char*>(saved) + round_up(static_cast<size_t>(n) * vpad * 2, 256));
-  FwdSaveEpilogue::Params p{targets, n, v, vpad, n_tiles, inv_t * kLog2e, inv_t, part, zy, u, ref};
-  return launch_gemm<FwdSaveEpilogue, false, false>(a, b, splits, p, dyn, status, stream);
+  if (part_e) {
+    KeepEpilogue<true>::Params p{targets, zy, n, v, vpad, inv_t * kLog2e, inv_t, part_s, part_e,
+                                 static_cast<__nv_bfloat16*>(q)};
+    return launch_gemm<KeepEpilogue<true>, false, false>(a, b, splits, p, dyn, status, stream);
+  }
+  KeepEpilogue<false>::Params p{targets, zy, n, v, vpad, inv_t * kLog2e, inv_t, part_s, nullptr,
+                                static_cast<__nv_bfloat16*>(q)};
+  return launch_gemm<KeepEpilogue<false>, false, false>(a, b, splits, p, dyn, status, stream);
 }
 
 size_t lmhead_tc_bwd_ws_bytes(long long chunk_rows, long long /*n*/, int /*h*/, int v) {
@@ -921,7 +890,7 @@ int lmhead_bwd_tc(const void* hidden_, const void* w_, const int32_t* targets, c
     A3PO_RETURN_IF((launch_gemm<DzEpilogue, false, false>(Operand{hid_c, nc, h, h}, Operand{w, v, h, h}, 0, dp,
                                                           dyn_m, status, stream)));
     // grad_hidden[t, j] = sum_v dz[t, v] W[v, j]:  A = dz (K = v contiguous), B = W read N-major
-    StoreBf16Epilogue::Params hp{grad_hidden + r0 * h, h, nc, h};
+    StoreBf16Epilogue::Params hp{grad_hidden + r0 * h, h, nc, h, nullptr};
     A3PO_RETURN_IF((launch_gemm<StoreBf16Epilogue, false, true>(Operand{dz, nc, v, vpad}, Operand{w, h, v, h}, 0, hp,
                                                                 dyn_m, status, stream)));
     // grad_w[v, j] (+)= sum_t dz[t, v] hidden[t, j]:  A = dz read M-major, B = hidden read N-major (K = t)
@@ -932,27 +901,41 @@ int lmhead_bwd_tc(const void* hidden_, const void* w_, const int32_t* targets, c
   return A3PO_OK;
 }
 
-// The two contractions of the backward on a dz matrix that already exists for all n rows
-// (built from saved logits): grad_hidden = dz W, grad_w (+)= dz^T hidden.
-int lmhead_bwd_from_dz_tc(const void* hidden_, const void* w_, const void* dz_, long long n, int h, int v,
-                          void* grad_hidden_, float* grad_w, int accumulate, const int* dyn_rows, uint32_t* status,
-                          cudaStream_t stream) {
-  const __nv_bfloat16* hidden = static_cast<const __nv_bfloat16*>(hidden_);
+// The two contractions of the backward on kept probability ratios q [n, v^8] (rows of one launch of the
+// keeping forward, `dyn_offset` rows into the compact row space whose size is *dyn_rows):
+//   grad_hidden[r, :] = row_scale[r] * sum_v q[r, v] W[v, :]
+//   grad_w[v, :]    (+)= sum_r q[r, v] hs[r, :]                 hs = row_scale * hidden, made by the caller
+// which equal dz W and dz^T hidden for dz[r, v] = row_scale[r] q[r, v].
+int lmhead_grad_hidden_from_kept_tc(const void* q_, const void* w_, const float* row_scale, long long n, int h, int v,
+                                    void* grad_hidden_, const int* dyn_rows, long long dyn_offset, uint32_t* status,
+                                    cudaStream_t stream) {
+  const __nv_bfloat16* q = static_cast<const __nv_bfloat16*>(q_);
   const __nv_bfloat16* w = static_cast<const __nv_bfloat16*>(w_);
-  const __nv_bfloat16* dz = static_cast<const __nv_bfloat16*>(dz_);
   const int vpad = static_cast<int>(round_up(static_cast<size_t>(v), 8));
   DynRows dyn_m;
   dyn_m.rows = dyn_rows;
+  dyn_m.offset = dyn_offset;
   dyn_m.cap = n;
-  DynRows dyn_k = dyn_m;
+  StoreBf16Epilogue::Params hp{static_cast<__nv_bfloat16*>(grad_hidden_), h, n, h, row_scale};
+  return launch_gemm<StoreBf16Epilogue, false, true>(Operand{q, n, v, vpad}, Operand{w, h, v, h}, 0, hp, dyn_m,
+                                                     status, stream);
+}
+
+int lmhead_grad_w_from_kept_tc(const void* q_, const void* hs_, long long n, int h, int v, float* grad_w,
+                               int accumulate, int zero_when_empty, const int* dyn_rows, long long dyn_offset,
+                               uint32_t* status, cudaStream_t stream) {
+  const __nv_bfloat16* q = static_cast<const __nv_bfloat16*>(q_);
+  const __nv_bfloat16* hs = static_cast<const __nv_bfloat16*>(hs_);
+  const int vpad = static_cast<int>(round_up(static_cast<size_t>(v), 8));
+  DynRows dyn_k;
+  dyn_k.rows = dyn_rows;
+  dyn_k.offset = dyn_offset;
+  dyn_k.cap = n;
   dyn_k.is_k = 1;
-  dyn_k.zero_when_empty = accumulate ? 0 : 1;
-  StoreBf16Epilogue::Params hp{static_cast<__nv_bfloat16*>(grad_hidden_), h, n, h};
-  A3PO_RETURN_IF((launch_gemm<StoreBf16Epilogue, false, true>(Operand{dz, n, v, vpad}, Operand{w, h, v, h}, 0, hp,
-                                                              dyn_m, status, stream)));
+  dyn_k.zero_when_empty = zero_when_empty;
   StoreF32Epilogue::Params wp{grad_w, h, v, h, accumulate ? 1 : 0};
-  return launch_gemm<StoreF32Epilogue, true, true>(Operand{dz, v, n, vpad}, Operand{hidden, h, n, h}, 0, wp, dyn_k,
-                                                   status, stream);
+  return launch_gemm<StoreF32Epilogue, true, true>(Operand{q, v, n, vpad}, Operand{hs, h, n, h}, 0, wp, dyn_k, status,
+                                                   stream);
 }
 
 }  // namespace a3po

@@ -7,13 +7,24 @@
 // the mask), two groups in flight per iteration; reductions go thread -> warp shuffle -> block
 // -> per-block partial -> one finalising block, in a fixed order, so results do not change from
 // run to run.
+//
+// An ABI call is ONE launch where the device allows it: the kernel is launched cooperatively and
+// runs up to three phases separated by grid-wide barriers: count the mask (when the backward needs
+// M and no forward statistics supply it), stream the tokens, and let block 0 sum the block
+// partials in index order.  Where a cooperative launch is not possible (or not wanted: the
+// static-scratch entry) the same phases run as separate launches.
+
+#include <cooperative_groups.h>
 
 #include <mutex>
 
 #include "a3po_common.cuh"
+#include "lmhead_internal.cuh"
 
 namespace a3po {
 namespace {
+
+namespace cg = cooperative_groups;
 
 constexpr int kLossThreads = 256;
 constexpr int kBlocksPerSm = 4;   // resident blocks per SM at <= 64 registers per thread
@@ -42,6 +53,16 @@ struct LossArgs {
   const float* grad_loss;        // device scalar or null
   const long long* n_valid_ptr;  // device: M, for the backward coefficient
   float* grad_logp;
+};
+
+// Phases a cooperative launch of loss_kernel runs besides the token stream.
+enum : int { kPhaseCountMask = 1, kPhaseFinalize = 2 };
+struct LossPhases {
+  int bits;
+  long long* block_counts;  // kPhaseCountMask: per-block mask counts, then M in n_valid
+  long long* n_valid;
+  float* loss;              // kPhaseFinalize outputs
+  a3po_stats* stats;
 };
 
 enum : int { kFwd = 0, kBwd = 1, kFwdBwd = 2 };
@@ -130,60 +151,10 @@ __device__ __forceinline__ void single(long long t, const LossArgs& p, float coe
   if (MODE != kFwd) p.grad_logp[t] = gr;
 }
 
-// VEC = true needs 16-byte aligned fp32/int32 arrays and a 4-byte aligned mask.
-template <int MODE, bool VEC, bool EXPLICIT>
-__global__ void __launch_bounds__(kLossThreads, kBlocksPerSm) loss_kernel(LossArgs p, LossPartial* partials) {
-  float coef = 0.f;
-  if (MODE != kFwd) {
-    long long m = *p.n_valid_ptr;
-    float gl = p.grad_loss ? *p.grad_loss : 1.0f;
-    coef = (m > 0) ? -gl / static_cast<float>(m) : 0.f;
-  }
-  Acc acc;
-  const long long tid = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
-  const long long nthreads = static_cast<long long>(gridDim.x) * blockDim.x;
-  if (VEC) {
-    const long long groups = p.n >> 2;
-    long long g = tid;
-    for (; g + nthreads < groups; g += 2 * nthreads) {
-      group4<MODE, EXPLICIT>(g, p, coef, acc);
-      group4<MODE, EXPLICIT>(g + nthreads, p, coef, acc);
-    }
-    if (g < groups) group4<MODE, EXPLICIT>(g, p, coef, acc);
-    const long long t = (groups << 2) + tid;  // ragged tail: at most three tokens
-    if (t < p.n) single<MODE, EXPLICIT>(t, p, coef, acc);
-  } else {
-    for (long long t = tid; t < p.n; t += nthreads) single<MODE, EXPLICIT>(t, p, coef, acc);
-  }
-  if (MODE == kBwd) return;
-
-  double sum = warp_sum(acc.sum);
-  long long nv = warp_sum(static_cast<long long>(acc.n_valid));
-  long long nc = warp_sum(static_cast<long long>(acc.n_clipped));
-  float mx = warp_max(acc.iw_max);
-  float mn = warp_min(acc.iw_min);
-  __shared__ LossPartial sh[kLossThreads / kWarp];
-  const int lane = threadIdx.x % kWarp, warp = threadIdx.x / kWarp;
-  if (lane == 0) sh[warp] = LossPartial{sum, nv, nc, mx, mn};
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    LossPartial out = sh[0];
-    for (int w = 1; w < kLossThreads / kWarp; ++w) {
-      out.sum += sh[w].sum;
-      out.n_valid += sh[w].n_valid;
-      out.n_clipped += sh[w].n_clipped;
-      out.iw_max = fmaxf(out.iw_max, sh[w].iw_max);
-      out.iw_min = fminf(out.iw_min, sh[w].iw_min);
-    }
-    partials[blockIdx.x] = out;
-  }
-}
-
-// Sums the per-block partials in a fixed order: loss = -sum / max(M,1), plus the diagnostics.
-__global__ void __launch_bounds__(kLossThreads) loss_finalize_kernel(const LossPartial* partials,
-                                                                    int count, float* loss,
-                                                                    a3po_stats* stats) {
-  __shared__ LossPartial sh[kLossThreads];
+// Sums `count` per-block partials in a fixed order (every thread a strided subsequence, then a
+// shared-memory tree): loss = -sum / max(M,1), plus the diagnostics.  Called by one whole block.
+__device__ __forceinline__ void finalize_block(const LossPartial* partials, int count, float* loss,
+                                               a3po_stats* stats, LossPartial* sh /*[kLossThreads]*/) {
   LossPartial mine{0.0, 0, 0, 0.f, 3.4e38f};
   for (int i = threadIdx.x; i < count; i += kLossThreads) {
     const LossPartial q = partials[i];
@@ -218,9 +189,10 @@ __global__ void __launch_bounds__(kLossThreads) loss_finalize_kernel(const LossP
   }
 }
 
-// M = number of non-zero mask bytes.  16 mask bytes per load where alignment allows.
-__global__ void __launch_bounds__(kLossThreads) mask_count_kernel(const uint8_t* mask, long long n,
-                                                                 long long* block_counts) {
+// This block's share of M = number of non-zero mask bytes (16 mask bytes per load where alignment
+// allows); the block total goes to block_counts[blockIdx.x].
+__device__ __forceinline__ void count_mask_block(const uint8_t* mask, long long n, long long* block_counts,
+                                                 long long* sh /*[kLossThreads / kWarp]*/) {
   long long count = 0;
   const long long tid = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
   const long long nthreads = static_cast<long long>(gridDim.x) * blockDim.x;
@@ -237,7 +209,6 @@ __global__ void __launch_bounds__(kLossThreads) mask_count_kernel(const uint8_t*
   }
   for (long long t = done + tid; t < n; t += nthreads) count += mask[t] != 0;
   count = warp_sum(count);
-  __shared__ long long sh[kLossThreads / kWarp];
   if (threadIdx.x % kWarp == 0) sh[threadIdx.x / kWarp] = count;
   __syncthreads();
   if (threadIdx.x == 0) {
@@ -247,9 +218,9 @@ __global__ void __launch_bounds__(kLossThreads) mask_count_kernel(const uint8_t*
   }
 }
 
-__global__ void __launch_bounds__(kLossThreads) mask_count_finalize_kernel(const long long* block_counts,
-                                                                          int count, long long* out) {
-  __shared__ long long sh[kLossThreads];
+// Sum of `count` block counts in a fixed order; called by one whole block.
+__device__ __forceinline__ void sum_counts_block(const long long* block_counts, int count, long long* out,
+                                                 long long* sh /*[kLossThreads]*/) {
   long long mine = 0;
   for (int i = threadIdx.x; i < count; i += kLossThreads) mine += block_counts[i];
   sh[threadIdx.x] = mine;
@@ -259,6 +230,89 @@ __global__ void __launch_bounds__(kLossThreads) mask_count_finalize_kernel(const
     __syncthreads();
   }
   if (threadIdx.x == 0) *out = sh[0];
+}
+
+// VEC = true needs 16-byte aligned fp32/int32 arrays and a 4-byte aligned mask.
+// ph.bits != 0 only in a cooperative launch (the grid-wide barriers are legal there and nowhere else).
+template <int MODE, bool VEC, bool EXPLICIT>
+__global__ void __launch_bounds__(kLossThreads, kBlocksPerSm) loss_kernel(LossArgs p, LossPartial* partials,
+                                                                          LossPhases ph) {
+  __shared__ LossPartial sh[kLossThreads];
+  if (ph.bits & kPhaseCountMask) {
+    long long* shc = reinterpret_cast<long long*>(sh);
+    count_mask_block(p.mask, p.n, ph.block_counts, shc);
+    cg::this_grid().sync();
+    if (blockIdx.x == 0) sum_counts_block(ph.block_counts, gridDim.x, ph.n_valid, shc);
+    cg::this_grid().sync();
+  }
+  float coef = 0.f;
+  if (MODE != kFwd) {
+    long long m = *reinterpret_cast<const volatile long long*>(p.n_valid_ptr);
+    float gl = p.grad_loss ? *p.grad_loss : 1.0f;
+    coef = (m > 0) ? -gl / static_cast<float>(m) : 0.f;
+  }
+  Acc acc;
+  const long long tid = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+  const long long nthreads = static_cast<long long>(gridDim.x) * blockDim.x;
+  if (VEC) {
+    const long long groups = p.n >> 2;
+    long long g = tid;
+    for (; g + nthreads < groups; g += 2 * nthreads) {
+      group4<MODE, EXPLICIT>(g, p, coef, acc);
+      group4<MODE, EXPLICIT>(g + nthreads, p, coef, acc);
+    }
+    if (g < groups) group4<MODE, EXPLICIT>(g, p, coef, acc);
+    const long long t = (groups << 2) + tid;  // ragged tail: at most three tokens
+    if (t < p.n) single<MODE, EXPLICIT>(t, p, coef, acc);
+  } else {
+    for (long long t = tid; t < p.n; t += nthreads) single<MODE, EXPLICIT>(t, p, coef, acc);
+  }
+  if (MODE == kBwd) return;
+
+  double sum = warp_sum(acc.sum);
+  long long nv = warp_sum(static_cast<long long>(acc.n_valid));
+  long long nc = warp_sum(static_cast<long long>(acc.n_clipped));
+  float mx = warp_max(acc.iw_max);
+  float mn = warp_min(acc.iw_min);
+  const int lane = threadIdx.x % kWarp, warp = threadIdx.x / kWarp;
+  __syncthreads();   // the count phase may have used the shared array
+  if (lane == 0) sh[warp] = LossPartial{sum, nv, nc, mx, mn};
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    LossPartial out = sh[0];
+    for (int w = 1; w < kLossThreads / kWarp; ++w) {
+      out.sum += sh[w].sum;
+      out.n_valid += sh[w].n_valid;
+      out.n_clipped += sh[w].n_clipped;
+      out.iw_max = fmaxf(out.iw_max, sh[w].iw_max);
+      out.iw_min = fminf(out.iw_min, sh[w].iw_min);
+    }
+    partials[blockIdx.x] = out;
+  }
+  if (ph.bits & kPhaseFinalize) {
+    cg::this_grid().sync();
+    if (blockIdx.x == 0) finalize_block(partials, gridDim.x, ph.loss, ph.stats, sh);
+  }
+}
+
+// The same phases as separate launches.
+__global__ void __launch_bounds__(kLossThreads) loss_finalize_kernel(const LossPartial* partials,
+                                                                    int count, float* loss,
+                                                                    a3po_stats* stats) {
+  __shared__ LossPartial sh[kLossThreads];
+  finalize_block(partials, count, loss, stats, sh);
+}
+
+__global__ void __launch_bounds__(kLossThreads) mask_count_kernel(const uint8_t* mask, long long n,
+                                                                 long long* block_counts) {
+  __shared__ long long sh[kLossThreads / kWarp];
+  count_mask_block(mask, n, block_counts, sh);
+}
+
+__global__ void __launch_bounds__(kLossThreads) mask_count_finalize_kernel(const long long* block_counts,
+                                                                          int count, long long* out) {
+  __shared__ long long sh[kLossThreads];
+  sum_counts_block(block_counts, count, out, sh);
 }
 
 // versions given per sequence: write the per-token array the streaming kernels read.
@@ -287,20 +341,49 @@ size_t loss_ws_bytes(long long n) {
          256 + round_up(sizeof(int32_t) * static_cast<size_t>(n > 0 ? n : 0), 256) + 256;
 }
 
-int grid_for(long long n_items) {
+int grid_for(long long n_items, int max_blocks = kMaxLossBlocks) {
   long long want = (n_items + kLossThreads - 1) / kLossThreads;
   long long cap = static_cast<long long>(sm_count()) * kBlocksPerSm;
-  if (cap > kMaxLossBlocks) cap = kMaxLossBlocks;
+  if (cap > max_blocks) cap = max_blocks;
   if (want > cap) want = cap;
   if (want < 1) want = 1;
   return static_cast<int>(want);
 }
 
+using LossKernel = void (*)(LossArgs, LossPartial*, LossPhases);
+
+LossKernel pick_kernel(int mode, bool vec, bool explicit_anchor) {
+#define A3PO_PICK(MODE)                                                                  \
+  (explicit_anchor ? (vec ? loss_kernel<MODE, true, true> : loss_kernel<MODE, false, true>) \
+                   : (vec ? loss_kernel<MODE, true, false> : loss_kernel<MODE, false, false>))
+  if (mode == kFwd) return A3PO_PICK(kFwd);
+  if (mode == kBwd) return A3PO_PICK(kBwd);
+  return A3PO_PICK(kFwdBwd);
+#undef A3PO_PICK
+}
+
+// Largest grid of `kernel` whose blocks are all resident at once on the current device (what a
+// cooperative launch requires); 0 if the device cannot launch cooperatively.
+int cooperative_capacity(LossKernel kernel) {
+  int dev = -1, coop = 0, per_sm = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess || !coop ||
+      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kLossThreads, 0) != cudaSuccess) {
+    cudaGetLastError();
+    return 0;
+  }
+  return per_sm * sm_count();
+}
+
+int kernel_id_of(int mode) { return mode == kFwd ? kKLossFwd : (mode == kBwd ? kKLossBwd : kKLossFwdBwd); }
+
+// allow_single_launch = false keeps every phase in its own plain launch.
 int run_loss(int mode, const float* logp, const float* behav, const float* prox, const int32_t* versions,
              int versions_per_seq,
              const int32_t* cu_seqlens, int b, int32_t current_version, const float* adv, const uint8_t* mask,
              long long n, float clip_eps, int detach, const float* grad_loss, const a3po_stats* fwd_stats,
-             float* loss, a3po_stats* stats, float* grad_logp, void* ws, size_t ws_bytes, void* stream_) {
+             float* loss, a3po_stats* stats, float* grad_logp, void* ws, size_t ws_bytes, void* stream_,
+             bool allow_single_launch = true) {
   if (n < 0 || !(clip_eps >= 0.f)) return A3PO_ERR_INVALID_ARG;
   if (n > 0 && (!logp || !behav || (!versions && !prox) || !adv || !mask)) return A3PO_ERR_INVALID_ARG;
   if (mode != kBwd && !loss) return A3PO_ERR_INVALID_ARG;
@@ -338,36 +421,46 @@ int run_loss(int mode, const float* logp, const float* behav, const float* prox,
   p.grad_loss = grad_loss;
   p.grad_logp = grad_logp;
   p.n_valid_ptr = nullptr;
-
-  if (mode != kFwd) {
-    if (fwd_stats) {
-      p.n_valid_ptr = reinterpret_cast<const long long*>(&fwd_stats->n_valid);
-    } else {
-      const int cb = grid_for((n + 15) / 16);
-      A3PO_LAUNCH(kKMaskCount, stream, mask_count_kernel<<<cb, kLossThreads, 0, stream>>>(mask, n, w.block_counts));
-      A3PO_RETURN_IF(after_launch());
-      A3PO_LAUNCH(kKMaskCountFinalize, stream,
-                  mask_count_finalize_kernel<<<1, kLossThreads, 0, stream>>>(w.block_counts, cb, w.n_valid));
-      A3PO_RETURN_IF(after_launch());
-      p.n_valid_ptr = w.n_valid;
-    }
-  }
+  const bool need_count = mode != kFwd && !fwd_stats;
+  if (mode != kFwd) p.n_valid_ptr = fwd_stats ? reinterpret_cast<const long long*>(&fwd_stats->n_valid) : w.n_valid;
 
   const bool vec = aligned_to(logp, 16) && aligned_to(behav, 16) && aligned_to(versions, 16) && aligned_to(prox, 16) &&
                    aligned_to(adv, 16) && aligned_to(mask, 4) && (mode == kFwd || aligned_to(grad_logp, 16));
-  const int blocks = grid_for(vec ? (n + 7) / 8 : n);
-#define A3PO_LAUNCH_LOSS(MODE, KID)                                                                        \
-  do {                                                                                                     \
-    if (prox) {                                                                                            \
-      if (vec) A3PO_LAUNCH(KID, stream, (loss_kernel<MODE, true, true><<<blocks, kLossThreads, 0, stream>>>(p, w.partials)));   \
-      else A3PO_LAUNCH(KID, stream, (loss_kernel<MODE, false, true><<<blocks, kLossThreads, 0, stream>>>(p, w.partials)));      \
-    } else if (vec) A3PO_LAUNCH(KID, stream, (loss_kernel<MODE, true, false><<<blocks, kLossThreads, 0, stream>>>(p, w.partials))); \
-    else A3PO_LAUNCH(KID, stream, (loss_kernel<MODE, false, false><<<blocks, kLossThreads, 0, stream>>>(p, w.partials)));       \
-  } while (0)
-  if (mode == kFwd) A3PO_LAUNCH_LOSS(kFwd, kKLossFwd);
-  else if (mode == kBwd) A3PO_LAUNCH_LOSS(kBwd, kKLossBwd);
-  else A3PO_LAUNCH_LOSS(kFwdBwd, kKLossFwdBwd);
-#undef A3PO_LAUNCH_LOSS
+  LossKernel kernel = pick_kernel(mode, vec, prox != nullptr);
+  int blocks = grid_for(vec ? (n + 7) / 8 : n);
+  LossPhases ph{0, w.block_counts, w.n_valid, loss, stats};
+  if (need_count) ph.bits |= kPhaseCountMask;
+  if (mode != kBwd) ph.bits |= kPhaseFinalize;
+
+  // ---- one cooperative launch: [count the mask] -> stream -> [sum the partials]
+  if (ph.bits != 0 && allow_single_launch) {
+    const int cap = cooperative_capacity(kernel);
+    if (cap >= 1) {
+      if (blocks > cap) blocks = cap;
+      void* kargs[] = {&p, &w.partials, &ph};
+      cudaError_t err;
+      {
+        ProfileScope scope(kernel_id_of(mode), stream);
+        err = cudaLaunchCooperativeKernel(reinterpret_cast<void*>(kernel), dim3(blocks), dim3(kLossThreads), kargs, 0,
+                                          stream);
+      }
+      if (err == cudaSuccess) return after_launch();
+      cudaGetLastError();  // not launchable this way here: fall through to the separate launches
+      blocks = grid_for(vec ? (n + 7) / 8 : n);
+    }
+  }
+
+  // ---- the same phases as separate launches
+  if (need_count) {
+    const int cb = grid_for((n + 15) / 16);
+    A3PO_LAUNCH(kKMaskCount, stream, mask_count_kernel<<<cb, kLossThreads, 0, stream>>>(mask, n, w.block_counts));
+    A3PO_RETURN_IF(after_launch());
+    A3PO_LAUNCH(kKMaskCountFinalize, stream,
+                mask_count_finalize_kernel<<<1, kLossThreads, 0, stream>>>(w.block_counts, cb, w.n_valid));
+    A3PO_RETURN_IF(after_launch());
+  }
+  ph.bits = 0;
+  A3PO_LAUNCH(kernel_id_of(mode), stream, (kernel<<<blocks, kLossThreads, 0, stream>>>(p, w.partials, ph)));
   A3PO_RETURN_IF(after_launch());
   if (mode != kBwd) {
     A3PO_LAUNCH(kKLossFinalize, stream,
@@ -378,6 +471,38 @@ int run_loss(int mode, const float* logp, const float* behav, const float* prox,
 }
 
 }  // namespace
+
+// ---- loss on a slice of tokens with M known, partials kept for a later finalize (row-chunked step)
+size_t loss_partial_bytes() { return sizeof(LossPartial); }
+int loss_max_partials() { return kMaxLossBlocks; }
+int loss_blocks_for(long long n, int max_blocks) { return grid_for((n + 7) / 8, max_blocks); }
+
+int loss_fwd_bwd_slice(const float* logp, const float* behav, const int32_t* versions, const float* adv,
+                       const uint8_t* mask, long long n, int32_t current_version, float clip_eps,
+                       const long long* n_valid, float* grad_logp, void* partials, int blocks, cudaStream_t stream) {
+  LossArgs p;
+  p.logp = logp; p.behav = behav; p.versions = versions; p.prox = nullptr; p.adv = adv; p.mask = mask; p.n = n;
+  p.current_version = current_version;
+  p.lo = 1.0f - clip_eps; p.hi = 1.0f + clip_eps;
+  p.detach = 1;
+  p.grad_loss = nullptr;
+  p.grad_logp = grad_logp;
+  p.n_valid_ptr = n_valid;
+  const bool vec = aligned_to(logp, 16) && aligned_to(behav, 16) && aligned_to(versions, 16) && aligned_to(adv, 16) &&
+                   aligned_to(mask, 4) && aligned_to(grad_logp, 16);
+  LossKernel kernel = pick_kernel(kFwdBwd, vec, false);
+  LossPhases ph{0, nullptr, nullptr, nullptr, nullptr};
+  A3PO_LAUNCH(kKLossFwdBwd, stream, (kernel<<<blocks, kLossThreads, 0, stream>>>(
+                                        p, static_cast<LossPartial*>(partials), ph)));
+  return after_launch();
+}
+
+int loss_finalize_partials(const void* partials, int count, float* loss, a3po_stats* stats, cudaStream_t stream) {
+  A3PO_LAUNCH(kKLossFinalize, stream, loss_finalize_kernel<<<1, kLossThreads, 0, stream>>>(
+                                          static_cast<const LossPartial*>(partials), count, loss, stats));
+  return after_launch();
+}
+
 }  // namespace a3po
 
 extern "C" {
@@ -449,7 +574,7 @@ int a3po_loss_fwd_static(const float* logp, const float* behav_logp, const int32
   A3PO_RETURN_IF(a3po::static_loss_scratch(&scratch));
   return a3po::run_loss(a3po::kFwd, logp, behav_logp, nullptr, versions, versions_per_seq, cu_seqlens, B, current_version,
                         adv, mask, N, clip_eps, 1, nullptr, nullptr, loss, stats, nullptr, scratch,
-                        a3po::kStaticScratchBytes, stream);
+                        a3po::kStaticScratchBytes, stream, /*allow_single_launch=*/false);
 }
 
 int a3po_loss_bwd(const float* logp, const float* behav_logp, const int32_t* versions, int versions_per_seq,

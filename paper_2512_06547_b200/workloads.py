@@ -74,6 +74,37 @@ def lm_head_operands(n, h, v, dtype, seed, device="cpu"):
     return hidden, w
 
 
+def peak_targets(hidden, w, rng, p_lo=0.3, p_hi=0.999, late_fraction=0.5):
+    """Turns flat random rows into confident ones, the way an RL fine-tuning batch looks (sampled tokens
+    mostly have high probability under the policy that is trained on them).
+
+    Every row t gets its own target y_t (all distinct), half of them (late_fraction) in the last eighth of
+    the vocabulary so that they fall into late column tiles and the last vocabulary split, and W[y_t] is
+    moved along hidden[t] by the amount that lifts the target's logit to about
+    ln V + 1/2 + logit(P_t) with P_t log-uniform in odds between p_lo and p_hi: the target probability
+    then lands near P_t (the other V - 1 logits stay ~ N(0,1), whose log-sum-exp is ln V + 1/2).
+    Modifies `w` in place (same dtype, rounded RNE) and returns the int32 targets [N] (numpy)."""
+    n, h = hidden.shape
+    v = w.shape[0]
+    if n > v:
+        raise ValueError("peak_targets needs at most V rows (targets are distinct)")
+    n_late = min(int(n * late_fraction), max(v // 8, 1))
+    late_pool = np.arange(v - max(v // 8, 1), v)
+    late = rng.choice(late_pool, size=n_late, replace=False)
+    rest_pool = np.setdiff1d(np.arange(v), late, assume_unique=False)
+    rest = rng.choice(rest_pool, size=n - n_late, replace=False)
+    targets = np.concatenate([late, rest]).astype(np.int32)
+    rng.shuffle(targets)
+    odds = np.exp(rng.uniform(np.log(p_lo / (1 - p_lo)), np.log(p_hi / (1 - p_hi)), size=n))
+    lift = torch.from_numpy((np.log(v) + 0.5 + np.log(odds)).astype(np.float32)).to(hidden.device)
+    hid = hidden.float()
+    y = torch.from_numpy(targets.astype(np.int64)).to(hidden.device)
+    base = (hid * w[y].float()).sum(dim=1)                       # the target's logit before the nudge
+    step = ((lift - base) / (hid * hid).sum(dim=1).clamp_min(1e-6)).unsqueeze(1) * hid
+    w[y] = (w[y].float() + step).to(w.dtype)
+    return targets
+
+
 def group_normalised_advantages(rewards, group_size, norm_eps=1e-6):
     """GRPO-style advantage, one per sequence: (R - mean_group) / (std_group + norm_eps)."""
     r = np.asarray(rewards, dtype=np.float64).reshape(-1, group_size)

@@ -194,7 +194,7 @@ def test_forward_keep_backward_kept_pair_matches_oracle_and_plain_pair():
     mask_np = (rng.random(n) < 0.7).astype(np.uint8)
     mask = torch.from_numpy(mask_np).to(DEV)
     g = g * mask                                                # skipped rows carry no gradient
-    kept = a3po.new_workspace(a3po.a3po_kept_logits_bytes(n, v))
+    kept = a3po.new_workspace(a3po.a3po_kept_bytes(n, v))
     ws = a3po.new_workspace(max(a3po.a3po_token_logprobs_fwd_keep_workspace_bytes(n, h, v),
                                 a3po.a3po_token_logprobs_bwd_kept_workspace_bytes(n, h, v)))
     logp, lse = torch.full((n,), 5.0, device=DEV), torch.full((n,), 5.0, device=DEV)
@@ -225,6 +225,6 @@ def test_forward_keep_backward_kept_pair_matches_oracle_and_plain_pair():
     h_odd, w_odd, t_odd, g_odd = _problem(16, 12, 40, "bf16", 93)
     with pytest.raises(a3po.A3poError) as e:
         a3po.a3po_token_logprobs_fwd_keep(h_odd, w_odd, t_odd, torch.empty(16, device=DEV), torch.empty(16, device=DEV),
-                                          a3po.new_workspace(a3po.a3po_kept_logits_bytes(16, 40)),
+                                          a3po.new_workspace(a3po.a3po_kept_bytes(16, 40)),
                                           a3po.new_workspace(a3po.a3po_token_logprobs_fwd_keep_workspace_bytes(16, 12, 40)))
     assert e.value.code == -2
