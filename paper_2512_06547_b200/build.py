@@ -1,11 +1,15 @@
 """Builds liba3po.so (sm_100a) from csrc/*.cu with nvcc; no GPU needed to compile.
 
-    python -m paper_2512_06547_b200.build [--force] [--verbose]
+    python -m paper_2512_06547_b200.build [--force] [--verbose] [--tuning]
 
 Each translation unit is compiled to an object file in parallel, then linked into
 paper_2512_06547_b200/lib/liba3po.so (statically linked CUDA runtime; the driver API is
 reached through the runtime's entry-point lookup, so the library loads on machines without
 libcuda).  Objects are rebuilt only when a source or header is newer.
+
+--tuning builds a second library, lib/liba3po_tuning.so, with -DA3PO_TUNING: the same code plus
+environment overrides of a few scheduling constants and a per-CTA trace of the GEMM kernels, for
+sweeps and profiling.  The package never loads it.
 """
 from __future__ import annotations
 
@@ -46,19 +50,22 @@ def _headers():
     return hs
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
+def build(force: bool = False, verbose: bool = False, tuning: bool = False) -> str:
     nvcc = _nvcc()
-    os.makedirs(OBJ_DIR, exist_ok=True)
+    obj_dir = OBJ_DIR + ("_tuning" if tuning else "")
+    lib_path = os.path.join(LIB_DIR, "liba3po_tuning.so") if tuning else LIB_PATH
+    extra = ["-DA3PO_TUNING"] if tuning else []
+    os.makedirs(obj_dir, exist_ok=True)
     os.makedirs(LIB_DIR, exist_ok=True)
     newest_header = max(os.path.getmtime(h) for h in _headers())
     jobs = []
     objs = []
     for src in _sources():
-        obj = os.path.join(OBJ_DIR, os.path.basename(src)[:-3] + ".o")
+        obj = os.path.join(obj_dir, os.path.basename(src)[:-3] + ".o")
         objs.append(obj)
         stale = force or not os.path.exists(obj) or os.path.getmtime(obj) < max(os.path.getmtime(src), newest_header)
         if stale:
-            cmd = [nvcc, *ARCH_FLAGS, *COMMON, "-c", src, "-o", obj]
+            cmd = [nvcc, *ARCH_FLAGS, *COMMON, *extra, "-c", src, "-o", obj]
             if verbose:
                 cmd.insert(1, "-Xptxas")
                 cmd.insert(2, "-v")
@@ -74,18 +81,19 @@ def build(force: bool = False, verbose: bool = False) -> str:
                 sys.stderr.write(" ".join(cmd) + "\n" + res.stdout + res.stderr)
             if res.returncode != 0:
                 raise RuntimeError(f"nvcc failed on {cmd[-3]}")
-    if jobs or force or not os.path.exists(LIB_PATH):
-        link = [nvcc, *ARCH_FLAGS, "-shared", "-Xcompiler", "-fPIC", "-o", LIB_PATH, *objs, "-cudart", "static"]
+    if jobs or force or not os.path.exists(lib_path):
+        link = [nvcc, *ARCH_FLAGS, "-shared", "-Xcompiler", "-fPIC", "-o", lib_path, *objs, "-cudart", "static"]
         res = subprocess.run(link, capture_output=True, text=True)
         if res.returncode != 0:
             sys.stderr.write(res.stdout + res.stderr)
             raise RuntimeError("link failed")
-    return LIB_PATH
+    return lib_path
 
 
 if __name__ == "__main__":
     ap = argparse.ArgumentParser()
     ap.add_argument("--force", action="store_true")
     ap.add_argument("--verbose", action="store_true")
+    ap.add_argument("--tuning", action="store_true")
     a = ap.parse_args()
-    print(build(force=a.force, verbose=a.verbose))
+    print(build(force=a.force, verbose=a.verbose, tuning=a.tuning))

@@ -30,7 +30,7 @@ int sm_count();
 enum KernelId : int {
   kKLossFwd = 0, kKLossBwd, kKLossFwdBwd, kKLossFinalize, kKMaskCount, kKMaskCountFinalize, kKExpandVersions,
   kKMergePartials, kKSimtFwd, kKSimtDz, kKSimtGemm, kKTcFwd, kKTcDz, kKTcGradHidden, kKTcGradW, kKCompact, kKGrpo,
-  kKSelfTest, kKTcFwdKeep, kKKeptRows, kKH2D,
+  kKSelfTest, kKTcFwdKeep, kKKeptRows, kKH2D, kKMoveRows,
   kKernelIdCount
 };
 

@@ -224,7 +224,7 @@ const char* a3po_kernel_name(int kernel_id) {
       "loss_fwd", "loss_bwd", "loss_fwd_bwd", "loss_finalize", "mask_count", "mask_count_finalize",
       "expand_versions", "merge_partials", "lmhead_fwd_fp32pipe", "lmhead_dz_fp32pipe", "gemm_fp32pipe",
       "gemm_tn<fwd_logsoftmax>", "gemm_tn<dz>", "gemm_tn<grad_hidden>", "gemm_tn<grad_w>", "compact_rows", "grpo_advantages", "selftest",
-      "gemm_tn<fwd_logsoftmax+keep>", "kept_rows", "h2d_copies"};
+      "gemm_tn<fwd_logsoftmax+keep>", "kept_rows", "h2d_copies", "move_kept_rows"};
   return (kernel_id >= 0 && kernel_id < kKernelIdCount) ? names[kernel_id] : "?";
 }
 
@@ -547,8 +547,8 @@ int a3po_token_logprobs_bwd_kept(const void* hidden, const void* w, const int32_
   if (!arena.ok()) return A3PO_ERR_WORKSPACE;
 
   // the target's entry of q and the per-row factor of dz, then the two contractions on q itself
-  A3PO_RETURN_IF(prepare_kept_backward(count, 0, cap, H, V, inv_temperature, sprime, targets_c, nullptr, grad_logp,
-                                       idx, nullptr, hidden, row_scale, q, hs, stream));
+  A3PO_RETURN_IF(prepare_kept_backward(count, 0, cap, nullptr, nullptr, H, V, inv_temperature, sprime, targets_c,
+                                       nullptr, grad_logp, idx, nullptr, hidden, row_scale, nullptr, q, hs, stream));
   A3PO_RETURN_IF(lmhead_grad_hidden_from_kept_tc(q, w, row_scale, cap, H, V, ghc, count, 0, status, stream));
   A3PO_RETURN_IF(scatter_rows(ghc, H, pos, N, grad_hidden, stream));
   return lmhead_grad_w_from_kept_tc(q, hs, cap, H, V, grad_w, accumulate_grad_w, accumulate_grad_w ? 0 : 1, count, 0,
@@ -566,10 +566,10 @@ constexpr int kStepMaxSplits = 64;
 // Workspace of the step that keeps the forward's softmax for the backward, one chunk of compact rows at a time.
 struct StepLayout {
   // whole batch
-  size_t count, scan, pos, idx, targets_c, hidden_c, zy, sprime, logp_c, lse_c, g_c, ent_c, behav_c, adv_c, row_scale,
+  size_t count, scan, pos, idx, targets_c, hidden_c, zy, sprime, logp_c, lse_c, g_c, ent_c, behav_c, adv_c,
       versions_c, mask_c, n_valid, partials;
   // one chunk
-  size_t part_s, part_e, q, hs, ghc;
+  size_t part_s, part_e, q, hs, ghc, perm, move_src, move_dst, bwd_idx, scale_p, bwd_count;
   size_t total;
 };
 StepLayout step_layout(long long n, int h, int v, long long chunk_rows) {
@@ -587,7 +587,7 @@ StepLayout step_layout(long long n, int h, int v, long long chunk_rows) {
   s.hidden_c = take(cap * static_cast<size_t>(h) * 2);
   s.zy = take(4 * cap); s.sprime = take(4 * cap); s.logp_c = take(4 * cap); s.lse_c = take(4 * cap);
   s.g_c = take(4 * cap); s.ent_c = take(4 * cap); s.behav_c = take(4 * cap); s.adv_c = take(4 * cap);
-  s.row_scale = take(4 * cap); s.versions_c = take(4 * cap);
+  s.versions_c = take(4 * cap);
   s.mask_c = take(cap);
   s.n_valid = take(sizeof(long long));
   s.partials = take(loss_partial_bytes() * loss_max_partials());
@@ -596,6 +596,9 @@ StepLayout step_layout(long long n, int h, int v, long long chunk_rows) {
   s.q = take(lmhead_tc_kept_bytes(chunk_rows, v));
   s.hs = take(rc * static_cast<size_t>(h) * 2);
   s.ghc = take(rc * static_cast<size_t>(h) * 2);
+  s.perm = take(4 * rc); s.move_src = take(4 * rc); s.move_dst = take(4 * rc); s.bwd_idx = take(4 * rc);
+  s.scale_p = take(4 * rc);
+  s.bwd_count = take(2 * sizeof(int));   // rows of the chunk's backward, rows moved to make them contiguous
   s.total = off;
   return s;
 }
@@ -690,7 +693,12 @@ int a3po_train_step(const void* hidden, const int32_t* targets, const float* beh
   auto f32 = [&](size_t off) { return reinterpret_cast<float*>(base + off); };
   float *zy = f32(lay.zy), *sprime = f32(lay.sprime), *logp_c = f32(lay.logp_c), *lse_c = f32(lay.lse_c);
   float *g_c = f32(lay.g_c), *ent_c = f32(lay.ent_c), *behav_c = f32(lay.behav_c), *adv_c = f32(lay.adv_c);
-  float* row_scale = f32(lay.row_scale);
+  float* scale_p = f32(lay.scale_p);
+  int* perm = reinterpret_cast<int*>(base + lay.perm);
+  int* move_src = reinterpret_cast<int*>(base + lay.move_src);
+  int* move_dst = reinterpret_cast<int*>(base + lay.move_dst);
+  int* bwd_idx = reinterpret_cast<int*>(base + lay.bwd_idx);
+  int* bwd_count = reinterpret_cast<int*>(base + lay.bwd_count);
   int32_t* versions_c = reinterpret_cast<int32_t*>(base + lay.versions_c);
   uint8_t* mask_c = reinterpret_cast<uint8_t*>(base + lay.mask_c);
   long long* n_valid = reinterpret_cast<long long*>(base + lay.n_valid);
@@ -723,13 +731,16 @@ int a3po_train_step(const void* hidden, const int32_t* targets, const float* beh
                                       current_version, clip_eps, n_valid, g_c + c0,
                                       partials + static_cast<size_t>(i) * loss_blocks * loss_partial_bytes(),
                                       loss_blocks, stream));
-    A3PO_RETURN_IF(prepare_kept_backward(cb.count, c0, rows, H, V, inv_temperature, sprime, cb.targets_c, g_c, nullptr,
-                                         cb.idx, hidden_c, nullptr, row_scale, q, hs, stream));
-    A3PO_RETURN_IF(lmhead_grad_hidden_from_kept_tc(q, w, row_scale + c0, rows, H, V, ghc, cb.count, c0, status,
-                                                   stream));
-    A3PO_RETURN_IF(scatter_rows_range(ghc, H, cb.idx, cb.count, c0, rows, grad_hidden, stream));
+    // the backward's rows: those with a non-zero gradient (clipped tokens drop out), made contiguous in q
+    A3PO_RETURN_IF(plan_backward_rows(g_c, cb.count, c0, rows, bwd_count, bwd_count + 1, perm, move_src, move_dst, q,
+                                      V, stream));
+    A3PO_RETURN_IF(prepare_kept_backward(cb.count, c0, rows, bwd_count, perm, H, V, inv_temperature, sprime,
+                                         cb.targets_c, g_c, nullptr, cb.idx, hidden_c, nullptr, scale_p, bwd_idx, q, hs,
+                                         stream));
+    A3PO_RETURN_IF(lmhead_grad_hidden_from_kept_tc(q, w, scale_p, rows, H, V, ghc, bwd_count, 0, status, stream));
+    A3PO_RETURN_IF(scatter_rows_range(ghc, H, bwd_idx, bwd_count, rows, grad_hidden, stream));
     A3PO_RETURN_IF(lmhead_grad_w_from_kept_tc(q, hs, rows, H, V, grad_w, (accumulate_grad_w || i > 0) ? 1 : 0,
-                                              (i == 0 && !accumulate_grad_w) ? 1 : 0, cb.count, c0, status, stream));
+                                              (i == 0 && !accumulate_grad_w) ? 1 : 0, bwd_count, 0, status, stream));
   }
   A3PO_RETURN_IF(finish_batch_outputs(cb.pos, N, logp_c, logp, lse_c, lse, g_c, grad_logp, ent_c, entropy,
                                       grad_hidden, H, stream));

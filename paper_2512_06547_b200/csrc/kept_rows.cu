@@ -118,25 +118,117 @@ gather_loss_inputs_kernel(const int* __restrict__ idx, const int* __restrict__ c
   }
 }
 
-// One warp per row of the launch.
+// Which rows of a launch's range take part in the backward, and how to make them contiguous by moving as few
+// rows as possible.  Among the `live` rows of the range, K have a non-zero upstream gradient.  Positions
+// 0 .. K-1 are the backward's rows: a position whose own row has g != 0 keeps it (perm[p] = p); the others
+// ("holes", rows with g == 0: clipped tokens) are filled, in order, with the rows at positions >= K that
+// have g != 0.  Only those rows have to be copied (move_src[i] -> move_dst[i]); a stable compaction would
+// move almost every row.  One block; the sums involved are integer, so the plan is deterministic.
+constexpr int kPlanThreads = 1024;
+__global__ void __launch_bounds__(kPlanThreads)
+plan_backward_rows_kernel(const float* __restrict__ g_c, const int* __restrict__ count, long long offset,
+                          long long rows, int* __restrict__ bwd_count, int* __restrict__ n_moves,
+                          int* __restrict__ perm, int* __restrict__ move_src, int* __restrict__ move_dst) {
+  __shared__ int sh[kPlanThreads];
+  __shared__ int s_nz_before_k;
+  long long live = static_cast<long long>(*count) - offset;
+  live = live < 0 ? 0 : (live > rows ? rows : live);
+  const long long per = (live + kPlanThreads - 1) / kPlanThreads;
+  long long lo = static_cast<long long>(threadIdx.x) * per;
+  lo = lo > live ? live : lo;
+  const long long hi = (lo + per > live) ? live : lo + per;
+  const float* g = g_c + offset;
+  int nz = 0;
+  for (long long p = lo; p < hi; ++p) nz += (g[p] != 0.f) ? 1 : 0;
+  sh[threadIdx.x] = nz;
+  __syncthreads();
+  for (int off = 1; off < kPlanThreads; off <<= 1) {  // Hillis-Steele inclusive scan
+    const int add = (threadIdx.x >= off) ? sh[threadIdx.x - off] : 0;
+    __syncthreads();
+    sh[threadIdx.x] += add;
+    __syncthreads();
+  }
+  const int before = sh[threadIdx.x] - nz;   // non-zero rows in front of this thread's segment
+  const long long k = sh[kPlanThreads - 1];  // rows of the backward
+  if (threadIdx.x == 0) s_nz_before_k = static_cast<int>(k);  // stands when no position >= k exists
+  __syncthreads();
+  if (lo <= k && k < hi) {                   // this segment holds position k: non-zero rows in front of it
+    int c = before;
+    for (long long p = lo; p < k; ++p) c += (g[p] != 0.f) ? 1 : 0;
+    s_nz_before_k = c;
+  }
+  __syncthreads();
+  const int nz_before_k = s_nz_before_k;
+  int running = before;
+  for (long long p = lo; p < hi; ++p) {
+    const bool is_nz = g[p] != 0.f;
+    if (p < k) {
+      if (is_nz) perm[p] = static_cast<int>(p);
+      else move_dst[p - running] = static_cast<int>(p);        // the (p - running)-th hole
+    } else if (is_nz) {
+      move_src[running - nz_before_k] = static_cast<int>(p);   // the matching filler
+    }
+    running += is_nz ? 1 : 0;
+  }
+  __threadfence_block();
+  __syncthreads();
+  const int holes = static_cast<int>(k) - nz_before_k;
+  for (int i = threadIdx.x; i < holes; i += kPlanThreads) perm[move_dst[i]] = move_src[i];
+  if (threadIdx.x == 0) {
+    *bwd_count = static_cast<int>(k);
+    *n_moves = holes;
+  }
+}
+
+// q[move_dst[i], :] = q[move_src[i], :] for the planned moves (rows of one launch, pitch vpad).
+constexpr int kMoveCols = kRowThreads * 8 * 2;   // columns per block iteration: two 16-byte pieces per thread
 __global__ void __launch_bounds__(kRowThreads)
-prepare_kept_backward_kernel(const int* __restrict__ count, long long offset, long long rows, int h, int v,
+move_rows_kernel(__nv_bfloat16* __restrict__ q, long long vpad, const int* __restrict__ move_src,
+                 const int* __restrict__ move_dst, const int* __restrict__ n_moves) {
+  const int moves = *n_moves;
+  const int segs = static_cast<int>((vpad + kMoveCols - 1) / kMoveCols);
+  const long long items = static_cast<long long>(moves) * segs;
+  for (long long item = blockIdx.x; item < items; item += gridDim.x) {
+    const int i = static_cast<int>(item / segs);
+    const long long col_a = static_cast<long long>(item % segs) * kMoveCols + threadIdx.x * 8;
+    const long long col_b = col_a + kRowThreads * 8;
+    const __nv_bfloat16* src = q + static_cast<long long>(move_src[i]) * vpad;
+    __nv_bfloat16* dst = q + static_cast<long long>(move_dst[i]) * vpad;
+    uint4 a = make_uint4(0u, 0u, 0u, 0u), b = a;
+    if (col_a < vpad) a = __ldcs(reinterpret_cast<const uint4*>(src + col_a));
+    if (col_b < vpad) b = __ldcs(reinterpret_cast<const uint4*>(src + col_b));
+    if (col_a < vpad) *reinterpret_cast<uint4*>(dst + col_a) = a;
+    if (col_b < vpad) *reinterpret_cast<uint4*>(dst + col_b) = b;
+  }
+}
+
+// One warp per position of the launch.
+__global__ void __launch_bounds__(kRowThreads)
+prepare_kept_backward_kernel(const int* __restrict__ count, long long offset, long long rows,
+                             const int* __restrict__ bwd_count, const int* __restrict__ perm, int h, int v,
                              long long vpad, float inv_t, const float* __restrict__ sprime,
                              const int32_t* __restrict__ targets_c, const float* __restrict__ g_c,
                              const float* __restrict__ g_batch, const int* __restrict__ idx,
                              const __nv_bfloat16* __restrict__ hidden_c, const __nv_bfloat16* __restrict__ hidden_batch,
-                             float* __restrict__ row_scale, __nv_bfloat16* __restrict__ q,
+                             float* __restrict__ row_scale, int* __restrict__ bwd_idx, __nv_bfloat16* __restrict__ q,
                              __nv_bfloat16* __restrict__ hs) {
-  const long long kept = *count;
-  const long long live = touched_rows(count, offset, rows);
+  long long k;   // positions that hold a row of the backward
+  if (bwd_count) {
+    k = *bwd_count;
+  } else {
+    k = static_cast<long long>(*count) - offset;
+    k = k < 0 ? 0 : (k > rows ? rows : k);
+  }
+  long long live = (k + 127) / 128 * 128;   // the GEMMs read whole 128-row tiles
+  live = live > rows ? rows : live;
   const int lane = threadIdx.x % kWarp;
   const long long warps = static_cast<long long>(gridDim.x) * kWarpsPerBlock;
   const int vec = h / 8;
-  for (long long r = static_cast<long long>(blockIdx.x) * kWarpsPerBlock + threadIdx.x / kWarp; r < live; r += warps) {
-    const long long c = offset + r;
-    uint4* dst = reinterpret_cast<uint4*>(hs + r * h);
+  for (long long p = static_cast<long long>(blockIdx.x) * kWarpsPerBlock + threadIdx.x / kWarp; p < live; p += warps) {
+    uint4* dst = reinterpret_cast<uint4*>(hs + p * h);
     float a = 0.f;
-    if (c < kept) {
+    if (p < k) {
+      const long long c = offset + (perm ? perm[p] : p);   // compact row that sits at this position
       const long long t = idx[c];
       const float g = g_c ? g_c[c] : g_batch[t];
       const float s = sprime[c];
@@ -144,7 +236,8 @@ prepare_kept_backward_kernel(const int* __restrict__ count, long long offset, lo
       if (!(fabsf(a) < 3.0e38f)) a = 0.f;   // a row the merge has flagged (non-finite sum): contributes nothing
       if (lane == 0) {
         const int y = min(max(targets_c[c], 0), v - 1);
-        q[r * vpad + y] = __float2bfloat16_rn(-s);
+        q[p * vpad + y] = __float2bfloat16_rn(-s);
+        if (bwd_idx) bwd_idx[p] = static_cast<int>(t);
       }
       const uint4* src = reinterpret_cast<const uint4*>(hidden_c ? hidden_c + c * h : hidden_batch + t * h);
       for (int j = lane; j < vec; j += kWarp) {
@@ -153,31 +246,29 @@ prepare_kept_backward_kernel(const int* __restrict__ count, long long offset, lo
         uint4 out;
         __nv_bfloat162* o = reinterpret_cast<__nv_bfloat162*>(&out);
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          const float2 f = __bfloat1622float2(x[k]);
-          o[k] = __floats2bfloat162_rn(a * f.x, a * f.y);
+        for (int e = 0; e < 4; ++e) {
+          const float2 f = __bfloat1622float2(x[e]);
+          o[e] = __floats2bfloat162_rn(a * f.x, a * f.y);
         }
         dst[j] = out;
       }
     } else {
       for (int j = lane; j < vec; j += kWarp) dst[j] = make_uint4(0u, 0u, 0u, 0u);
     }
-    if (lane == 0) row_scale[c] = a;
+    if (lane == 0) row_scale[p] = a;
   }
 }
 
 __global__ void __launch_bounds__(kRowThreads)
-scatter_rows_range_kernel(const __nv_bfloat16* __restrict__ src, int h, const int* __restrict__ idx,
-                          const int* __restrict__ count, long long offset, long long rows,
-                          __nv_bfloat16* __restrict__ dst) {
-  long long live = static_cast<long long>(*count) - offset;
-  live = live < 0 ? 0 : (live > rows ? rows : live);
+scatter_rows_range_kernel(const __nv_bfloat16* __restrict__ src, int h, const int* __restrict__ bwd_idx,
+                          const int* __restrict__ bwd_count, __nv_bfloat16* __restrict__ dst) {
+  const long long live = *bwd_count;
   const int lane = threadIdx.x % kWarp;
   const long long warps = static_cast<long long>(gridDim.x) * kWarpsPerBlock;
   const int vec = h / 8;
-  for (long long r = static_cast<long long>(blockIdx.x) * kWarpsPerBlock + threadIdx.x / kWarp; r < live; r += warps) {
-    const uint4* in = reinterpret_cast<const uint4*>(src + r * h);
-    uint4* out = reinterpret_cast<uint4*>(dst + static_cast<long long>(idx[offset + r]) * h);
+  for (long long p = static_cast<long long>(blockIdx.x) * kWarpsPerBlock + threadIdx.x / kWarp; p < live; p += warps) {
+    const uint4* in = reinterpret_cast<const uint4*>(src + p * h);
+    uint4* out = reinterpret_cast<uint4*>(dst + static_cast<long long>(bwd_idx[p]) * h);
     for (int j = lane; j < vec; j += kWarp) out[j] = in[j];
   }
 }
@@ -195,13 +286,16 @@ finish_scalars_kernel(const int* __restrict__ pos, long long n, const float* __r
   if (d) d[t] = p >= 0 ? d_c[p] : 0.f;
 }
 
+// Rows of the batch that no backward row was scattered to: not kept by the forward, or zero upstream gradient.
 __global__ void __launch_bounds__(kRowThreads)
-zero_unkept_rows_kernel(const int* __restrict__ pos, long long n, int h, __nv_bfloat16* __restrict__ dst) {
+zero_unkept_rows_kernel(const int* __restrict__ pos, const float* __restrict__ g_c, long long n, int h,
+                        __nv_bfloat16* __restrict__ dst) {
   const int lane = threadIdx.x % kWarp;
   const long long warps = static_cast<long long>(gridDim.x) * kWarpsPerBlock;
   const int vec = h / 8;
   for (long long t = static_cast<long long>(blockIdx.x) * kWarpsPerBlock + threadIdx.x / kWarp; t < n; t += warps) {
-    if (pos[t] >= 0) continue;
+    const int c = pos[t];
+    if (c >= 0 && (g_c == nullptr || g_c[c] != 0.f)) continue;
     uint4* out = reinterpret_cast<uint4*>(dst + t * h);
     for (int j = lane; j < vec; j += kWarp) out[j] = make_uint4(0u, 0u, 0u, 0u);
   }
@@ -247,25 +341,37 @@ int gather_loss_inputs(const int* idx, const int* count, long long cap, const fl
   return after_launch();
 }
 
-int prepare_kept_backward(const int* count, long long offset, long long rows, int h, int v, float inv_t,
-                          const float* sprime, const int32_t* targets_c, const float* g_c, const float* g_batch,
-                          const int* idx, const void* hidden_c, const void* hidden_batch, float* row_scale, void* q,
-                          void* hs, cudaStream_t stream) {
+int plan_backward_rows(const float* g_c, const int* count, long long offset, long long rows, int* bwd_count,
+                       int* n_moves, int* perm, int* move_src, int* move_dst, void* q, int v, cudaStream_t stream) {
+  if (rows <= 0) return A3PO_OK;
+  A3PO_LAUNCH(kKKeptRows, stream, (plan_backward_rows_kernel<<<1, kPlanThreads, 0, stream>>>(
+                                      g_c, count, offset, rows, bwd_count, n_moves, perm, move_src, move_dst)));
+  A3PO_RETURN_IF(after_launch());
+  const long long vpad = static_cast<long long>(round_up(static_cast<size_t>(v), 8));
+  A3PO_LAUNCH(kKMoveRows, stream, (move_rows_kernel<<<sm_count() * 8, kRowThreads, 0, stream>>>(
+                                      static_cast<__nv_bfloat16*>(q), vpad, move_src, move_dst, n_moves)));
+  return after_launch();
+}
+
+int prepare_kept_backward(const int* count, long long offset, long long rows, const int* bwd_count, const int* perm,
+                          int h, int v, float inv_t, const float* sprime, const int32_t* targets_c, const float* g_c,
+                          const float* g_batch, const int* idx, const void* hidden_c, const void* hidden_batch,
+                          float* row_scale, int* bwd_idx, void* q, void* hs, cudaStream_t stream) {
   if (rows <= 0) return A3PO_OK;
   const long long vpad = static_cast<long long>(round_up(static_cast<size_t>(v), 8));
   A3PO_LAUNCH(kKKeptRows, stream, (prepare_kept_backward_kernel<<<row_grid(rows), kRowThreads, 0, stream>>>(
-                                      count, offset, rows, h, v, vpad, inv_t, sprime, targets_c, g_c, g_batch, idx,
-                                      static_cast<const __nv_bfloat16*>(hidden_c),
-                                      static_cast<const __nv_bfloat16*>(hidden_batch), row_scale,
+                                      count, offset, rows, bwd_count, perm, h, v, vpad, inv_t, sprime, targets_c, g_c,
+                                      g_batch, idx, static_cast<const __nv_bfloat16*>(hidden_c),
+                                      static_cast<const __nv_bfloat16*>(hidden_batch), row_scale, bwd_idx,
                                       static_cast<__nv_bfloat16*>(q), static_cast<__nv_bfloat16*>(hs))));
   return after_launch();
 }
 
-int scatter_rows_range(const void* src, int h, const int* idx, const int* count, long long offset, long long rows,
-                       void* dst, cudaStream_t stream) {
+int scatter_rows_range(const void* src, int h, const int* bwd_idx, const int* bwd_count, long long rows, void* dst,
+                       cudaStream_t stream) {
   if (rows <= 0) return A3PO_OK;
   A3PO_LAUNCH(kKKeptRows, stream, (scatter_rows_range_kernel<<<row_grid(rows), kRowThreads, 0, stream>>>(
-                                      static_cast<const __nv_bfloat16*>(src), h, idx, count, offset, rows,
+                                      static_cast<const __nv_bfloat16*>(src), h, bwd_idx, bwd_count,
                                       static_cast<__nv_bfloat16*>(dst))));
   return after_launch();
 }
@@ -280,7 +386,7 @@ int finish_batch_outputs(const int* pos, long long n, const float* logp_c, float
   A3PO_RETURN_IF(after_launch());
   if (grad_hidden) {
     A3PO_LAUNCH(kKKeptRows, stream, (zero_unkept_rows_kernel<<<row_grid(n), kRowThreads, 0, stream>>>(
-                                        pos, n, h, static_cast<__nv_bfloat16*>(grad_hidden))));
+                                        pos, g_c, n, h, static_cast<__nv_bfloat16*>(grad_hidden))));
     A3PO_RETURN_IF(after_launch());
   }
   return A3PO_OK;

@@ -92,20 +92,27 @@ int merge_kept(const float* part_s, const float* part_e, const float* zy, const 
 int gather_loss_inputs(const int* idx, const int* count, long long cap, const float* behav, const int32_t* versions,
                        const float* adv, float* behav_c, int32_t* versions_c, float* adv_c, uint8_t* mask_c,
                        long long* n_valid, cudaStream_t stream);
-// Prepares the two gradient contractions for rows [offset, offset + rows):
-//   row_scale[c] = -g / (T (1 + sprime[c]))     g = g_c[c], or g_batch[idx[c]] when g_c is null
-//   q[c - offset, y_c] = -sprime[c]              (the target's entry: 1 - 1/p_y)
-//   hs[c - offset, :]  = row_scale[c] * hidden row   (hidden_c[c], or hidden_batch[idx[c]] when hidden_c is null)
-// rows from *count to the next multiple of 128 get scale 0 and zero hs rows.
-int prepare_kept_backward(const int* count, long long offset, long long rows, int h, int v, float inv_t,
-                          const float* sprime, const int32_t* targets_c, const float* g_c, const float* g_batch,
-                          const int* idx, const void* hidden_c, const void* hidden_batch, float* row_scale, void* q,
-                          void* hs, cudaStream_t stream);
-// dst[idx[c], :] = src[c - offset, :] for compact rows c in [offset, min(offset + rows, *count)).
-int scatter_rows_range(const void* src, int h, const int* idx, const int* count, long long offset, long long rows,
-                       void* dst, cudaStream_t stream);
+// Chooses the backward's rows among rows [offset, offset + rows): those with g_c != 0, K of them (-> *bwd_count).
+// They are made contiguous at positions 0 .. K-1 of the launch's q by moving only the rows that fill the holes
+// left by rows with g_c == 0 (clipped tokens); perm[p] = row of the range now at position p.
+int plan_backward_rows(const float* g_c, const int* count, long long offset, long long rows, int* bwd_count,
+                       int* n_moves, int* perm, int* move_src, int* move_dst, void* q, int v, cudaStream_t stream);
+// Prepares the two gradient contractions for the positions p of a launch (K = *bwd_count of them, or every row
+// of [offset, offset + rows) below *count when bwd_count is null; c = offset + perm[p], or offset + p):
+//   row_scale[p] = -g / (T (1 + sprime[c]))      g = g_c[c], or g_batch[idx[c]] when g_c is null
+//   q[p, y_c]    = -sprime[c]                     (the target's entry: 1 - 1/p_y)
+//   hs[p, :]     = row_scale[p] * hidden row      (hidden_c[c], or hidden_batch[idx[c]] when hidden_c is null)
+//   bwd_idx[p]   = idx[c]                         (batch row; skipped when bwd_idx is null)
+// positions from K to the next multiple of 128 get scale 0 and zero hs rows.
+int prepare_kept_backward(const int* count, long long offset, long long rows, const int* bwd_count, const int* perm,
+                          int h, int v, float inv_t, const float* sprime, const int32_t* targets_c, const float* g_c,
+                          const float* g_batch, const int* idx, const void* hidden_c, const void* hidden_batch,
+                          float* row_scale, int* bwd_idx, void* q, void* hs, cudaStream_t stream);
+// dst[bwd_idx[p], :] = src[p, :] for positions p < *bwd_count.
+int scatter_rows_range(const void* src, int h, const int* bwd_idx, const int* bwd_count, long long rows, void* dst,
+                       cudaStream_t stream);
 // Batch-space outputs from compact ones: out[t] = pos[t] >= 0 ? in_c[pos[t]] : 0 for up to four arrays (null = skip),
-// and, when grad_hidden is given, zero rows of grad_hidden [n, h] for rows that were not kept.
+// and, when grad_hidden is given, zero rows of grad_hidden [n, h] for rows that were not kept or have g_c == 0.
 int finish_batch_outputs(const int* pos, long long n, const float* logp_c, float* logp, const float* lse_c, float* lse,
                          const float* g_c, float* grad_logp, const float* ent_c, float* entropy, void* grad_hidden,
                          int h, cudaStream_t stream);

@@ -40,16 +40,25 @@ using namespace ptx;
 constexpr int BM = 128;
 constexpr int BN = 256;
 constexpr int BK = 64;
-constexpr int kStages = 4;
 constexpr int kTcThreads = 192;
 constexpr int kEpiChunk = 32;
-constexpr uint32_t kABytes = BM * BK * 2;
+constexpr uint32_t kABytes = BM * BK * 2;   // one 128-row A tile
 constexpr uint32_t kBBytes = BN * BK * 2;
-constexpr uint32_t kStageBytes = kABytes + kBBytes;
 constexpr uint32_t kMnBlockBytes = 64 * BK * 2;  // one 64 (M/N) x 64 (k) box of an MN-major operand
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kSlabBytes = BM * 128;  // output staging slab: 128 rows x 128 bytes
-constexpr size_t kSmemBytes = 1024 /*alignment slack*/ + kStages * kStageBytes + 2 * kSlabBytes + 256 /*barriers*/;
+// MT = A tiles (of 128 rows) a CTA multiplies with each B tile.  MT = 1: a 128 x 256 output tile, two accumulators
+// in TMEM so that the epilogue of one tile overlaps the MMAs of the next, 4-stage ring.  MT = 2: a 256 x 256 output
+// tile (all 512 TMEM columns, one accumulator set, no epilogue overlap), 3-stage ring of 64 KB stages: a third fewer
+// operand bytes per flop out of L2 and shared memory, for the contractions whose epilogue is negligible (K = V or
+// K = rows, thousands of k-blocks per tile).
+template <int MT> struct TileCfg {
+  static constexpr int kStages = MT == 1 ? 4 : 3;
+  static constexpr int kAccStages = 2 / MT;
+  static constexpr uint32_t kAStage = MT * kABytes;
+  static constexpr uint32_t kStageBytes = kAStage + kBBytes;
+  static constexpr size_t kSmemBytes = 1024 /*alignment slack*/ + kStages * kStageBytes + 2 * kSlabBytes + 256 /*barriers*/;
+};
 constexpr int kGroupM = 16;
 
 // Work decomposition: an item is (row tile, vocabulary split); a split is a contiguous range of
@@ -491,11 +500,26 @@ __device__ __forceinline__ bool all_epilogue_threads(bool pred) {
   return out != 0;
 }
 
+#ifdef A3PO_TUNING
+// Tuning builds only: per-CTA start / end of every GEMM launch in wall-clock nanoseconds and SM cycles, written to
+// a caller-provided buffer (a3po_tuning_set_trace), to read the finish-time spread of the CTAs and the SM clock a
+// kernel really ran at.
+struct TraceRecord {
+  unsigned long long t_begin_ns, t_end_ns, cycles, items;
+  // SM cycles each role spent waiting: producer on a free stage, MMA issuer on a filled stage, MMA issuer on a free
+  // accumulator, epilogue (warp 2) on a finished accumulator
+  unsigned long long wait_stage_free, wait_stage_full, wait_acc_free, wait_acc_full;
+};
+__device__ TraceRecord* g_trace = nullptr;
+__device__ unsigned int g_trace_capacity = 0;
+__device__ unsigned int g_trace_next = 0;
+#endif
+
 // ------------------------------------------------------------------------------------ the kernel
 // A_MN / B_MN: the operand is read from a tensor whose contiguous index is M (resp. N) instead of
 // K: it arrives as 64 x 64 boxes (64 M/N elements by 64 k) and is fed to the MMA as an MN-major
 // shared-memory matrix, so no transposed copy of the operand ever has to exist in memory.
-template <class Epi, bool A_MN, bool B_MN>
+template <class Epi, bool A_MN, bool B_MN, int MT>
 __global__ void __launch_bounds__(kTcThreads, 1)
 gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_c, ItemMap im_static, int k_blocks_static,
@@ -514,14 +538,19 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         else im.items = 0;
       }
     } else {
-      im.m_tiles = static_cast<int>((rows + BM - 1) / BM);
+      im.m_tiles = static_cast<int>((rows + BM * MT - 1) / (BM * MT));
       im.items = static_cast<long long>(im.m_tiles) * im.splits;
     }
   }
+  using Cfg = TileCfg<MT>;
+  constexpr int kStages = Cfg::kStages;
+  constexpr int kAccStages = Cfg::kAccStages;
+  constexpr uint32_t kAStage = Cfg::kAStage;
+  constexpr uint32_t kStageBytes = Cfg::kStageBytes;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* smem_a = smem;
-  uint8_t* smem_b = smem + kStages * kABytes;
+  uint8_t* smem_b = smem + kStages * kAStage;
   uint8_t* smem_slabs = smem + kStages * kStageBytes;  // two 16 KB output staging slabs
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem_slabs + 2 * kSlabBytes);
   uint64_t* empty_bar = full_bar + kStages;
@@ -532,13 +561,28 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
   const int warp = threadIdx.x / kWarp;
   const int lane = threadIdx.x % kWarp;
+#ifdef A3PO_TUNING
+  unsigned long long trace_t0 = 0, trace_c0 = 0;
+  __shared__ unsigned long long trace_wait[4];
+  unsigned long long waited = 0, waited2 = 0;
+  if (threadIdx.x == 0) {
+    trace_t0 = globaltimer_ns();
+    trace_c0 = static_cast<unsigned long long>(clock64());
+    trace_wait[0] = trace_wait[1] = trace_wait[2] = trace_wait[3] = 0;
+  }
+#define A3PO_TIMED_WAIT(acc, expr) [&] { const long long t_ = clock64(); const bool r_ = (expr); acc += clock64() - t_; return r_; }()
+#else
+#define A3PO_TIMED_WAIT(acc, expr) (expr)
+  constexpr int waited = 0, waited2 = 0;
+  (void)waited; (void)waited2;
+#endif
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < kStages; ++i) {
       mbar_init(&full_bar[i], 1);
       mbar_init(&empty_bar[i], 1);
     }
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < kAccStages; ++i) {
       mbar_init(&tmem_full_bar[i], 1);
       mbar_init(&tmem_empty_bar[i], 4);  // one arrival per epilogue warp
     }
@@ -570,16 +614,16 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const Item it = decode_item(im, i);
         for (int nt = it.n_begin; nt < it.n_end && ok; ++nt) {
           for (int kb = 0; kb < k_blocks; ++kb) {
-            if (!mbar_wait(&empty_bar[stage], phase ^ 1u, abort_flag)) { ok = false; break; }
+            if (!A3PO_TIMED_WAIT(waited, mbar_wait(&empty_bar[stage], phase ^ 1u, abort_flag))) { ok = false; break; }
             mbar_arrive_expect_tx(&full_bar[stage], kStageBytes);
-            uint8_t* sa = smem_a + stage * kABytes;
+            uint8_t* sa = smem_a + stage * kAStage;
             uint8_t* sb = smem_b + stage * kBBytes;
             if (A_MN) {
 #pragma unroll
-              for (int j = 0; j < BM / 64; ++j)
-                tma_load_2d(sa + j * kMnBlockBytes, &map_a, &full_bar[stage], it.m_tile * BM + j * 64, kb * BK);
+              for (int j = 0; j < MT * BM / 64; ++j)
+                tma_load_2d(sa + j * kMnBlockBytes, &map_a, &full_bar[stage], it.m_tile * (BM * MT) + j * 64, kb * BK);
             } else {
-              tma_load_2d(sa, &map_a, &full_bar[stage], kb * BK, it.m_tile * BM);
+              tma_load_2d(sa, &map_a, &full_bar[stage], kb * BK, it.m_tile * (BM * MT));  // one box of MT * 128 rows
             }
             if (B_MN) {
 #pragma unroll
@@ -608,24 +652,28 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       for (long long i = blockIdx.x; i < im.items && ok; i += gridDim.x) {
         const Item it = decode_item(im, i);
         for (int nt = it.n_begin; nt < it.n_end && ok; ++nt) {
-          if (!mbar_wait(&tmem_empty_bar[acc], acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+          if (!A3PO_TIMED_WAIT(waited2, mbar_wait(&tmem_empty_bar[acc], acc_phase ^ 1u, abort_flag))) { ok = false; break; }
           tcgen05_fence_after_sync();
-          const uint32_t tmem_d = tmem_base + static_cast<uint32_t>(acc * BN);
+          const uint32_t tmem_d = tmem_base + static_cast<uint32_t>(acc * BN * MT);
           for (int kb = 0; kb < k_blocks; ++kb) {
-            if (!mbar_wait(&full_bar[stage], phase, abort_flag)) { ok = false; break; }
+            if (!A3PO_TIMED_WAIT(waited, mbar_wait(&full_bar[stage], phase, abort_flag))) { ok = false; break; }
             tcgen05_fence_after_sync();
-            const uint32_t sa = smem_u32(smem_a + stage * kABytes);
+            const uint32_t sa = smem_u32(smem_a + stage * kAStage);
             const uint32_t sb = smem_u32(smem_b + stage * kBBytes);
             const uint64_t desc_a = A_MN ? umma_desc_mn_major_sw128(sa, kMnBlockBytes) : umma_desc_k_major_sw128(sa);
             const uint64_t desc_b = B_MN ? umma_desc_mn_major_sw128(sb, kMnBlockBytes) : umma_desc_k_major_sw128(sb);
 #pragma unroll
-            for (int k = 0; k < BK / 16; ++k)
-              umma_bf16(tmem_d, desc_a + a_step * k, desc_b + b_step * k, idesc, (kb | k) != 0 ? 1u : 0u);
+            for (int k = 0; k < BK / 16; ++k) {
+#pragma unroll
+              for (int mt = 0; mt < MT; ++mt)   // the A tiles of a stage lie kABytes apart (either major-ness)
+                umma_bf16(tmem_d + static_cast<uint32_t>(mt * BN), desc_a + mt * (kABytes >> 4) + a_step * k,
+                          desc_b + b_step * k, idesc, (kb | k) != 0 ? 1u : 0u);
+            }
             umma_commit(&empty_bar[stage]);  // stage reusable once these MMAs have read it
             if (++stage == kStages) { stage = 0; phase ^= 1u; }
           }
           if (ok) umma_commit(&tmem_full_bar[acc]);
-          if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+          if (++acc == kAccStages) { acc = 0; acc_phase ^= 1u; }
         }
       }
     }
@@ -644,40 +692,55 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     st.issuer = (threadIdx.x == 2 * kWarp);
     for (long long i = blockIdx.x; i < im.items && ok; i += gridDim.x) {
       const Item it = decode_item(im, i);
-      const int tile_row0 = it.m_tile * BM;
-      epi.begin(ep, static_cast<long long>(tile_row0) + row_in_tile);
+      const int item_row0 = it.m_tile * (BM * MT);
+      if (MT == 1) epi.begin(ep, static_cast<long long>(item_row0) + row_in_tile);
       for (int nt = it.n_begin; nt < it.n_end && ok; ++nt) {
         // the four epilogue warps share named barriers further down: they must agree on giving up
         if (!zero_output) {
-          ok = all_epilogue_threads(mbar_wait(&tmem_full_bar[acc], acc_phase, abort_flag));
+          ok = all_epilogue_threads(A3PO_TIMED_WAIT(waited, mbar_wait(&tmem_full_bar[acc], acc_phase, abort_flag)));
           if (!ok) break;
           tcgen05_fence_after_sync();
         }
-        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(acc * BN);
 #pragma unroll 1
-        for (int c = 0; c < BN / kEpiChunk; ++c) {
-          uint32_t r[kEpiChunk];
-          if (!zero_output) {
-            tmem_ld_32x32(taddr + static_cast<uint32_t>(c * kEpiChunk), r);
-            tmem_ld_wait();
-          } else {
+        for (int mt = 0; mt < MT; ++mt) {
+          const int tile_row0 = item_row0 + mt * BM;
+          // epilogues of the MT = 2 kernels keep no state from one column tile to the next
+          if (MT > 1) epi.begin(ep, static_cast<long long>(tile_row0) + row_in_tile);
+          const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
+                                 static_cast<uint32_t>(acc * BN * MT + mt * BN);
+#pragma unroll 1
+          for (int c = 0; c < BN / kEpiChunk; ++c) {
+            uint32_t r[kEpiChunk];
+            if (!zero_output) {
+              tmem_ld_32x32(taddr + static_cast<uint32_t>(c * kEpiChunk), r);
+              tmem_ld_wait();
+            } else {
 #pragma unroll
-            for (int j = 0; j < kEpiChunk; ++j) r[j] = 0u;
+              for (int j = 0; j < kEpiChunk; ++j) r[j] = 0u;
+            }
+            epi.chunk(ep, tile_row0, nt * BN + c * kEpiChunk, r, st);
           }
-          epi.chunk(ep, tile_row0, nt * BN + c * kEpiChunk, r, st);
         }
         if (!zero_output) {
           tcgen05_fence_before_sync();
           __syncwarp();
           if (lane == 0) mbar_arrive(&tmem_empty_bar[acc]);
-          if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+          if (++acc == kAccStages) { acc = 0; acc_phase ^= 1u; }
         }
       }
-      if (ok) epi.end(ep, static_cast<long long>(tile_row0) + row_in_tile, it.split);
+      if (MT == 1 && ok) epi.end(ep, static_cast<long long>(item_row0) + row_in_tile, it.split);
     }
     st.drain();  // shared memory must stay valid until the copy engine has read every submitted slab
   }
 
+#ifdef A3PO_TUNING
+  if (lane == 0 || (warp < 2)) {
+    if (warp == 0 && waited) trace_wait[0] = waited;
+    if (warp == 1 && waited) trace_wait[1] = waited;
+    if (warp == 1 && waited2) trace_wait[2] = waited2;
+    if (warp == 2 && lane == 0) trace_wait[3] = waited;
+  }
+#endif
   if (!ok) {
     *abort_flag = 1;
     if (status) atomicOr(status, A3PO_STATUS_WAIT_TIMEOUT);
@@ -689,6 +752,19 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     tcgen05_fence_after_sync();
     tmem_dealloc(tmem_base, kTmemCols);
   }
+#ifdef A3PO_TUNING
+  if (threadIdx.x == 0 && g_trace != nullptr) {
+    const unsigned int slot = atomicAdd(&g_trace_next, 1u);
+    if (slot < g_trace_capacity) {
+      unsigned long long mine = 0;
+      for (long long i = blockIdx.x; i < im.items; i += gridDim.x) ++mine;
+      g_trace[slot] = TraceRecord{trace_t0, globaltimer_ns(), static_cast<unsigned long long>(clock64()) - trace_c0,
+                                  (static_cast<unsigned long long>(Epi::kKernelId) << 48) |
+                                      (static_cast<unsigned long long>(blockIdx.x) << 32) | mine,
+                                  trace_wait[0], trace_wait[1], trace_wait[2], trace_wait[3]};
+    }
+  }
+#endif
 }
 
 // ------------------------------------------------------------------------------------ host side
@@ -741,15 +817,16 @@ struct DynRows {
 };
 
 // C[M, N] = sum_k A[m, k] B[n, k];  splits = 0 means one column tile per work item.
-template <class Epi, bool A_MN, bool B_MN>
+template <class Epi, bool A_MN, bool B_MN, int MT = 1>
 int launch_gemm(const Operand& a, const Operand& b, int splits, const typename Epi::Params& ep, const DynRows& dyn,
                 uint32_t* status, cudaStream_t stream) {
+  constexpr size_t kSmemBytes = TileCfg<MT>::kSmemBytes;
   CUtensorMap map_a, map_b, map_c;
-  A3PO_RETURN_IF(make_map(&map_a, a, A_MN, BM));
+  A3PO_RETURN_IF(make_map(&map_a, a, A_MN, BM * MT));
   A3PO_RETURN_IF(make_map(&map_b, b, B_MN, BN));
   A3PO_RETURN_IF(Epi::make_c_map(ep, &map_c));
   ItemMap im;
-  im.m_tiles = static_cast<int>((a.mn_extent + BM - 1) / BM);
+  im.m_tiles = static_cast<int>((a.mn_extent + BM * MT - 1) / (BM * MT));
   im.n_tiles = static_cast<int>((b.mn_extent + BN - 1) / BN);
   im.splits = splits > 0 ? splits : im.n_tiles;
   im.items = static_cast<long long>(im.m_tiles) * im.splits;
@@ -760,7 +837,7 @@ int launch_gemm(const Operand& a, const Operand& b, int splits, const typename E
   im.dyn_offset = dyn.offset;
   im.dyn_cap = dyn.cap;
   const int k_blocks = static_cast<int>((a.k_extent + BK - 1) / BK);
-  auto kernel = gemm_tn_kernel<Epi, A_MN, B_MN>;
+  auto kernel = gemm_tn_kernel<Epi, A_MN, B_MN, MT>;
   if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemBytes)) !=
       cudaSuccess) {
     cudaGetLastError();
@@ -774,6 +851,14 @@ int launch_gemm(const Operand& a, const Operand& b, int splits, const typename E
   return after_launch();
 }
 
+// The gradient contractions take the 256 x 256 tile (MT = 2); a tuning build can fall back to 128 x 256 for A/B runs.
+template <class Epi, bool A_MN, bool B_MN>
+int launch_grad_gemm(const Operand& a, const Operand& b, const typename Epi::Params& ep, const DynRows& dyn,
+                     uint32_t* status, cudaStream_t stream) {
+  if (tuning_override("A3PO_GRAD_MT", 2) == 1) return launch_gemm<Epi, A_MN, B_MN, 1>(a, b, 0, ep, dyn, status, stream);
+  return launch_gemm<Epi, A_MN, B_MN, 2>(a, b, 0, ep, dyn, status, stream);
+}
+
 // Scratch of the backward: one bf16 dz chunk [chunk_rows, vpad].
 size_t bwd_ws_layout(long long chunk_rows, int v) {
   const size_t vpad = round_up(static_cast<size_t>(v), 8);
@@ -781,6 +866,29 @@ size_t bwd_ws_layout(long long chunk_rows, int v) {
 }
 
 }  // namespace
+
+#ifdef A3PO_TUNING
+}  // namespace a3po
+// Tuning builds only (not part of the ABI in include/): where the GEMM kernels record their per-CTA trace.
+// `records` is a device buffer of `capacity` 64-byte records, or null to stop tracing; resets the write position.
+extern "C" int a3po_tuning_set_trace(void* records, unsigned int capacity) {
+  a3po::TraceRecord* p = static_cast<a3po::TraceRecord*>(records);
+  unsigned int zero = 0;
+  if (cudaMemcpyToSymbol(a3po::g_trace, &p, sizeof(p)) != cudaSuccess ||
+      cudaMemcpyToSymbol(a3po::g_trace_capacity, &capacity, sizeof(capacity)) != cudaSuccess ||
+      cudaMemcpyToSymbol(a3po::g_trace_next, &zero, sizeof(zero)) != cudaSuccess) {
+    cudaGetLastError();
+    return A3PO_ERR_CUDA;
+  }
+  return A3PO_OK;
+}
+extern "C" unsigned int a3po_tuning_trace_count() {
+  unsigned int n = 0;
+  if (cudaMemcpyFromSymbol(&n, a3po::g_trace_next, sizeof(n)) != cudaSuccess) cudaGetLastError();
+  return n;
+}
+namespace a3po {
+#endif
 
 // Exercises the bounded wait the pipelines rely on: a barrier nothing ever arrives at.
 int selftest_wait_timeout(uint32_t* status, unsigned timeout_ms, cudaStream_t stream) {
@@ -891,12 +999,12 @@ int lmhead_bwd_tc(const void* hidden_, const void* w_, const int32_t* targets, c
                                                           dyn_m, status, stream)));
     // grad_hidden[t, j] = sum_v dz[t, v] W[v, j]:  A = dz (K = v contiguous), B = W read N-major
     StoreBf16Epilogue::Params hp{grad_hidden + r0 * h, h, nc, h, nullptr};
-    A3PO_RETURN_IF((launch_gemm<StoreBf16Epilogue, false, true>(Operand{dz, nc, v, vpad}, Operand{w, h, v, h}, 0, hp,
-                                                                dyn_m, status, stream)));
+    A3PO_RETURN_IF((launch_grad_gemm<StoreBf16Epilogue, false, true>(Operand{dz, nc, v, vpad}, Operand{w, h, v, h}, hp,
+                                                                     dyn_m, status, stream)));
     // grad_w[v, j] (+)= sum_t dz[t, v] hidden[t, j]:  A = dz read M-major, B = hidden read N-major (K = t)
     StoreF32Epilogue::Params wp{grad_w, h, v, h, (accumulate || r0 > 0) ? 1 : 0};
-    A3PO_RETURN_IF((launch_gemm<StoreF32Epilogue, true, true>(Operand{dz, v, nc, vpad}, Operand{hid_c, h, nc, h}, 0,
-                                                              wp, dyn_k, status, stream)));
+    A3PO_RETURN_IF((launch_grad_gemm<StoreF32Epilogue, true, true>(Operand{dz, v, nc, vpad}, Operand{hid_c, h, nc, h},
+                                                                   wp, dyn_k, status, stream)));
   }
   return A3PO_OK;
 }
@@ -917,8 +1025,8 @@ int lmhead_grad_hidden_from_kept_tc(const void* q_, const void* w_, const float*
   dyn_m.offset = dyn_offset;
   dyn_m.cap = n;
   StoreBf16Epilogue::Params hp{static_cast<__nv_bfloat16*>(grad_hidden_), h, n, h, row_scale};
-  return launch_gemm<StoreBf16Epilogue, false, true>(Operand{q, n, v, vpad}, Operand{w, h, v, h}, 0, hp, dyn_m,
-                                                     status, stream);
+  return launch_grad_gemm<StoreBf16Epilogue, false, true>(Operand{q, n, v, vpad}, Operand{w, h, v, h}, hp, dyn_m,
+                                                          status, stream);
 }
 
 int lmhead_grad_w_from_kept_tc(const void* q_, const void* hs_, long long n, int h, int v, float* grad_w,
@@ -934,8 +1042,8 @@ int lmhead_grad_w_from_kept_tc(const void* q_, const void* hs_, long long n, int
   dyn_k.is_k = 1;
   dyn_k.zero_when_empty = zero_when_empty;
   StoreF32Epilogue::Params wp{grad_w, h, v, h, accumulate ? 1 : 0};
-  return launch_gemm<StoreF32Epilogue, true, true>(Operand{q, v, n, vpad}, Operand{hs, h, n, h}, 0, wp, dyn_k, status,
-                                                   stream);
+  return launch_grad_gemm<StoreF32Epilogue, true, true>(Operand{q, v, n, vpad}, Operand{hs, h, n, h}, wp, dyn_k,
+                                                        status, stream);
 }
 
 }  // namespace a3po

@@ -6,7 +6,7 @@ import torch
 import paper_2512_06547_b200 as a3po
 from oracle import a3po_oracle as orc
 from paper_2512_06547_b200 import workloads
-from tests.helpers import GRAD_FRO_RTOL, LOGP_TOL_BF16, LOGP_TOL_F32, rel_fro, to_np64
+from tests.helpers import GRAD_FRO_RTOL, LOGP_TOL_BF16, LOGP_TOL_F32, rel_fro, row_rel_err, to_np64
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
@@ -185,8 +185,64 @@ def test_masked_and_zero_gradient_rows_are_skipped_consistently():
         assert not to_np64(gh)[g_np == 0].any()
 
 
+def _keep_pair(hidden, w, targets, g, mask=None, want_entropy=False):
+    n, h = hidden.shape
+    v = w.shape[0]
+    kept = a3po.new_workspace(a3po.a3po_kept_bytes(n, v))
+    ws = a3po.new_workspace(max(a3po.a3po_token_logprobs_fwd_keep_workspace_bytes(n, h, v),
+                                a3po.a3po_token_logprobs_bwd_kept_workspace_bytes(n, h, v)))
+    logp, lse = torch.full((n,), 5.0, device=DEV), torch.full((n,), 5.0, device=DEV)
+    ent = torch.full((n,), 5.0, device=DEV) if want_entropy else None
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    a3po.a3po_token_logprobs_fwd_keep(hidden, w, targets, logp, lse, kept, ws, row_mask=mask, entropy=ent,
+                                      status=status)
+    ws.fill_(0xAB)                                              # the backward must not depend on the forward's scratch
+    gh = torch.full_like(hidden, 3.0)
+    gw = torch.full((v, h), 3.0, dtype=torch.float32, device=DEV)
+    a3po.a3po_token_logprobs_bwd_kept(hidden, w, targets, lse, g, kept, gh, gw, ws, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    return logp, lse, ent, gh, gw, kept, ws
+
+
+@pytest.mark.parametrize("n,h,v", [(600, 512, 8192 + 24), (300, 1536, 4096 + 40)])
+def test_peaked_rows_both_backward_paths(n, h, v):
+    """Confident rows, as in an RL fine-tuning batch: target probability between 0.3 and 0.999, half of the
+    targets in the last eighth of the vocabulary (late column tiles, last split).  dz at the target is
+    g (1 - p_y), a cancellation; the recomputing pair and the keeping pair must both hold the gradient
+    tolerance row by row, not only over the whole matrix."""
+    hidden, w, _, g = _problem(n, h, v, "bf16", 300 + n)
+    targets_np = workloads.peak_targets(hidden, w, np.random.default_rng(17 + n))
+    targets = torch.from_numpy(targets_np).to(DEV)
+    hn, wn = to_np64(hidden), to_np64(w)
+    logp_ref, lse_ref = orc.token_logprobs_fwd(hn, wn, targets_np)
+    p_y = np.exp(logp_ref)
+    assert p_y.min() < 0.45 and p_y.max() > 0.995 and np.median(p_y) > 0.8          # the rows really are peaked
+    gh_ref, gw_ref = orc.token_logprobs_bwd(hn, wn, targets_np, to_np64(g))
+    ent_ref = orc.token_entropy(hn, wn)
+    live = to_np64(g) != 0
+
+    logp, lse, ent, status = gpu_fwd(hidden, w, targets, want_entropy=True)
+    assert status == 0
+    gh, gw, status = gpu_bwd(hidden, w, targets, lse, g)
+    assert status == 0
+    k_logp, k_lse, k_ent, k_gh, k_gw, _, _ = _keep_pair(hidden, w, targets, g, want_entropy=True)
+    for tag, (lp, ls, en, a, b) in {"recomputing pair": (logp, lse, ent, gh, gw),
+                                    "keeping pair": (k_logp, k_lse, k_ent, k_gh, k_gw)}.items():
+        e_lp = np.max(np.abs(lp.cpu().numpy() - logp_ref))
+        e_ls = np.max(np.abs(ls.cpu().numpy() - lse_ref))
+        e_en = np.max(np.abs(en.cpu().numpy() - ent_ref))
+        e_row = row_rel_err(to_np64(a)[live], gh_ref[live])
+        e_gw = rel_fro(to_np64(b), gw_ref)
+        print(f"[peaked {tag} n={n} h={h} v={v}] logp {e_lp:.2e} lse {e_ls:.2e} entropy {e_en:.2e} "
+              f"grad_hidden rows: median {np.median(e_row):.2e} worst {e_row.max():.2e}  grad_w fro {e_gw:.2e}")
+        assert e_lp <= LOGP_TOL_BF16 and e_ls <= LOGP_TOL_BF16 and e_en <= 5e-3
+        assert e_row.max() <= GRAD_FRO_RTOL and e_gw <= GRAD_FRO_RTOL
+        assert not to_np64(a)[~live].any()
+
+
 def test_forward_keep_backward_kept_pair_matches_oracle_and_plain_pair():
-    """The forward that keeps its logits and the backward that uses them, as two separate calls with the
+    """The forward that keeps its softmax and the backward that uses it, as two separate calls with the
     upstream gradient computed in between (as under an autograd engine)."""
     n, h, v = 700, 512, 5000 + 24
     hidden, w, targets, g = _problem(n, h, v, "bf16", 91)
@@ -194,18 +250,7 @@ def test_forward_keep_backward_kept_pair_matches_oracle_and_plain_pair():
     mask_np = (rng.random(n) < 0.7).astype(np.uint8)
     mask = torch.from_numpy(mask_np).to(DEV)
     g = g * mask                                                # skipped rows carry no gradient
-    kept = a3po.new_workspace(a3po.a3po_kept_bytes(n, v))
-    ws = a3po.new_workspace(max(a3po.a3po_token_logprobs_fwd_keep_workspace_bytes(n, h, v),
-                                a3po.a3po_token_logprobs_bwd_kept_workspace_bytes(n, h, v)))
-    logp, lse = torch.full((n,), 5.0, device=DEV), torch.full((n,), 5.0, device=DEV)
-    status = torch.zeros(1, dtype=torch.int32, device=DEV)
-    a3po.a3po_token_logprobs_fwd_keep(hidden, w, targets, logp, lse, kept, ws, row_mask=mask, status=status)
-    ws.fill_(0xAB)                                              # the backward must not depend on the forward's scratch
-    gh = torch.full_like(hidden, 3.0)
-    gw = torch.full((v, h), 3.0, dtype=torch.float32, device=DEV)
-    a3po.a3po_token_logprobs_bwd_kept(hidden, w, targets, lse, g, kept, gh, gw, ws, status=status)
-    torch.cuda.synchronize()
-    assert int(status.item()) == 0
+    logp, lse, _, gh, gw, kept, ws = _keep_pair(hidden, w, targets, g, mask=mask)
     hn, wn, tn = to_np64(hidden), to_np64(w), targets.cpu().numpy()
     logp_ref, lse_ref = orc.token_logprobs_fwd(hn, wn, tn, row_mask=mask_np)
     assert np.max(np.abs(logp.cpu().numpy() - logp_ref)) <= LOGP_TOL_BF16
@@ -221,6 +266,15 @@ def test_forward_keep_backward_kept_pair_matches_oracle_and_plain_pair():
     a3po.a3po_token_logprobs_bwd_kept(hidden, w, targets, lse, g, kept, gh, acc, ws, accumulate_grad_w=True)
     torch.cuda.synchronize()
     assert rel_fro(to_np64(acc - base), gw_ref) <= GRAD_FRO_RTOL
+    # a row the forward skipped has nothing kept: whatever upstream gradient it carries is ignored (never used as
+    # an index), so the result is the one for g * mask
+    g_stray = g.clone()
+    g_stray[mask == 0] = 1.0
+    gh3 = torch.full_like(hidden, 3.0)
+    gw3 = torch.full((v, h), 3.0, dtype=torch.float32, device=DEV)
+    a3po.a3po_token_logprobs_bwd_kept(hidden, w, targets, lse, g_stray, kept, gh3, gw3, ws)
+    torch.cuda.synchronize()
+    assert torch.equal(gw3, gw) and torch.equal(gh3, gh)
     # shapes outside the tensor-core path are refused, not silently computed another way
     h_odd, w_odd, t_odd, g_odd = _problem(16, 12, 40, "bf16", 93)
     with pytest.raises(a3po.A3poError) as e:

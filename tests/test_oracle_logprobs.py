@@ -123,9 +123,18 @@ def _scalar_objective(hidden, w, targets, coeff, inv_t):
     return float(np.dot(coeff, logp))
 
 
-def test_backward_matches_finite_differences():
+@pytest.mark.parametrize("peaked", [False, True])
+def test_backward_matches_finite_differences(peaked):
     n, h, v = 5, 8, 17
     hidden, w, targets = _problem(n, h, v, 12)
+    if peaked:
+        # confident rows: the target's weight row is moved along the row's hidden state until the target holds
+        # most of the probability mass (p_y up to 0.999), where dz at the target, g (1 - p_y), is a cancellation
+        targets = np.arange(n) * 3 % v
+        for t, lift in enumerate([4.0, 6.0, 8.0, 10.0, 12.0]):
+            w[targets[t]] += lift * hidden[t] / np.dot(hidden[t], hidden[t])
+        p_y = np.exp(orc.token_logprobs_fwd(hidden, w, targets, inv_temperature=0.8)[0])
+        assert p_y.max() > 0.99 and np.median(p_y) > 0.5
     coeff = np.random.default_rng(13).standard_normal(n)
     inv_t = 0.8
     gh, gw = orc.token_logprobs_bwd(hidden, w, targets, coeff, inv_temperature=inv_t)
