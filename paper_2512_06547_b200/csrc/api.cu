@@ -443,7 +443,8 @@ size_t fwd_keep_ws_bytes(long long n, int h, int v) {
 
 size_t bwd_kept_ws_bytes(long long n, int h) {
   const size_t cap = static_cast<size_t>(compact_capacity(n));
-  return round_up(sizeof(float) * cap, 256) /*row_scale*/ + 2 * round_up(cap * static_cast<size_t>(h) * 2, 256) + 256;
+  return round_up(sizeof(float) * cap, 256) /*row_scale*/ + 2 * round_up(cap * static_cast<size_t>(h) * 2, 256) +
+         256 /*tile choice*/ + 256;
 }
 }  // namespace
 
@@ -544,12 +545,13 @@ int a3po_token_logprobs_bwd_kept(const void* hidden, const void* w, const int32_
   float* row_scale = arena.take<float>(static_cast<size_t>(cap));
   __nv_bfloat16* hs = arena.take<__nv_bfloat16>(static_cast<size_t>(cap) * H);
   __nv_bfloat16* ghc = arena.take<__nv_bfloat16>(static_cast<size_t>(cap) * H);
+  int* select = arena.take<int>(1);
   if (!arena.ok()) return A3PO_ERR_WORKSPACE;
 
   // the target's entry of q and the per-row factor of dz, then the two contractions on q itself
   A3PO_RETURN_IF(prepare_kept_backward(count, 0, cap, nullptr, nullptr, H, V, inv_temperature, sprime, targets_c,
                                        nullptr, grad_logp, idx, nullptr, hidden, row_scale, nullptr, q, hs, stream));
-  A3PO_RETURN_IF(lmhead_grad_hidden_from_kept_tc(q, w, row_scale, cap, H, V, ghc, count, 0, status, stream));
+  A3PO_RETURN_IF(lmhead_grad_hidden_from_kept_tc(q, w, row_scale, cap, H, V, ghc, count, 0, select, status, stream));
   A3PO_RETURN_IF(scatter_rows(ghc, H, pos, N, grad_hidden, stream));
   return lmhead_grad_w_from_kept_tc(q, hs, cap, H, V, grad_w, accumulate_grad_w, accumulate_grad_w ? 0 : 1, count, 0,
                                     status, stream);
@@ -566,10 +568,10 @@ constexpr int kStepMaxSplits = 64;
 // Workspace of the step that keeps the forward's softmax for the backward, one chunk of compact rows at a time.
 struct StepLayout {
   // whole batch
-  size_t count, scan, pos, idx, targets_c, hidden_c, zy, sprime, logp_c, lse_c, g_c, ent_c, behav_c, adv_c,
+  size_t count, scan, pos, idx, targets_c, zy, sprime, logp_c, lse_c, g_c, ent_c, behav_c, adv_c,
       versions_c, mask_c, n_valid, partials;
   // one chunk
-  size_t part_s, part_e, q, hs, ghc, perm, move_src, move_dst, bwd_idx, scale_p, bwd_count;
+  size_t hidden_c, part_s, part_e, q, hs, ghc, perm, move_src, move_dst, bwd_idx, scale_p, bwd_count;
   size_t total;
 };
 StepLayout step_layout(long long n, int h, int v, long long chunk_rows) {
@@ -584,13 +586,13 @@ StepLayout step_layout(long long n, int h, int v, long long chunk_rows) {
   s.pos = take(4 * rows);
   s.idx = take(4 * cap);
   s.targets_c = take(4 * cap);
-  s.hidden_c = take(cap * static_cast<size_t>(h) * 2);
   s.zy = take(4 * cap); s.sprime = take(4 * cap); s.logp_c = take(4 * cap); s.lse_c = take(4 * cap);
   s.g_c = take(4 * cap); s.ent_c = take(4 * cap); s.behav_c = take(4 * cap); s.adv_c = take(4 * cap);
   s.versions_c = take(4 * cap);
   s.mask_c = take(cap);
   s.n_valid = take(sizeof(long long));
   s.partials = take(loss_partial_bytes() * loss_max_partials());
+  s.hidden_c = take(rc * static_cast<size_t>(h) * 2);   // the chunk's rows of hidden, gathered
   s.part_s = take(4 * rc * kStepMaxSplits);
   s.part_e = take(4 * rc * kStepMaxSplits);
   s.q = take(lmhead_tc_kept_bytes(chunk_rows, v));
@@ -598,7 +600,7 @@ StepLayout step_layout(long long n, int h, int v, long long chunk_rows) {
   s.ghc = take(rc * static_cast<size_t>(h) * 2);
   s.perm = take(4 * rc); s.move_src = take(4 * rc); s.move_dst = take(4 * rc); s.bwd_idx = take(4 * rc);
   s.scale_p = take(4 * rc);
-  s.bwd_count = take(2 * sizeof(int));   // rows of the chunk's backward, rows moved to make them contiguous
+  s.bwd_count = take(4 * sizeof(int));   // rows of the chunk's backward, rows moved, tile choice of grad_hidden
   s.total = off;
   return s;
 }
@@ -714,7 +716,7 @@ int a3po_train_step(const void* hidden, const int32_t* targets, const float* beh
   if (max_blocks < 1) return A3PO_ERR_WORKSPACE;   // more than 4096 chunks: the workspace is far too small for N
   const int loss_blocks = loss_blocks_for(chunk_rows, max_blocks);
 
-  A3PO_RETURN_IF(compact_rows(hidden, H, targets, mask, nullptr, nullptr, N, cb, stream));
+  A3PO_RETURN_IF(compact_index(targets, mask, nullptr, nullptr, N, cb, stream));
   A3PO_RETURN_IF(gather_loss_inputs(cb.idx, cb.count, cap, behav_logp, versions, adv, behav_c, versions_c, adv_c,
                                     mask_c, n_valid, stream));
   A3PO_RETURN_IF(flag_bad_targets(targets, N, V, status, stream));
@@ -722,8 +724,9 @@ int a3po_train_step(const void* hidden, const int32_t* targets, const float* beh
     const long long c0 = static_cast<long long>(i) * chunk_rows;
     const long long rows = (c0 + chunk_rows <= cap) ? chunk_rows : cap - c0;
     const int splits = lmhead_tc_fwd_splits(rows, V);
+    A3PO_RETURN_IF(gather_rows_range(hidden, H, cb.idx, cb.count, c0, rows, cb.hidden_c, stream));
     A3PO_RETURN_IF(target_logits(hidden_c, w, cb.targets_c, cb.count, c0, rows, H, V, inv_temperature, zy, stream));
-    A3PO_RETURN_IF(lmhead_fwd_keep_tc(hidden_c + c0 * H, w, cb.targets_c + c0, zy + c0, rows, H, V, inv_temperature,
+    A3PO_RETURN_IF(lmhead_fwd_keep_tc(hidden_c, w, cb.targets_c + c0, zy + c0, rows, H, V, inv_temperature,
                                       splits, part_s, entropy ? part_e : nullptr, q, cb.count, c0, status, stream));
     A3PO_RETURN_IF(merge_kept(part_s, part_e, zy, cb.count, c0, rows, splits, inv_temperature, sprime, logp_c, lse_c,
                               entropy ? ent_c : nullptr, status, stream));
@@ -737,7 +740,8 @@ int a3po_train_step(const void* hidden, const int32_t* targets, const float* beh
     A3PO_RETURN_IF(prepare_kept_backward(cb.count, c0, rows, bwd_count, perm, H, V, inv_temperature, sprime,
                                          cb.targets_c, g_c, nullptr, cb.idx, hidden_c, nullptr, scale_p, bwd_idx, q, hs,
                                          stream));
-    A3PO_RETURN_IF(lmhead_grad_hidden_from_kept_tc(q, w, scale_p, rows, H, V, ghc, bwd_count, 0, status, stream));
+    A3PO_RETURN_IF(lmhead_grad_hidden_from_kept_tc(q, w, scale_p, rows, H, V, ghc, bwd_count, 0, bwd_count + 2, status,
+                                                   stream));
     A3PO_RETURN_IF(scatter_rows_range(ghc, H, bwd_idx, bwd_count, rows, grad_hidden, stream));
     A3PO_RETURN_IF(lmhead_grad_w_from_kept_tc(q, hs, rows, H, V, grad_w, (accumulate_grad_w || i > 0) ? 1 : 0,
                                               (i == 0 && !accumulate_grad_w) ? 1 : 0, bwd_count, 0, status, stream));

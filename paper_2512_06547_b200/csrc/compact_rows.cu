@@ -131,21 +131,23 @@ compact_fill_kernel(const uint8_t* __restrict__ row_mask, const float* __restric
 // partial tiles of the GEMMs see finite data.
 __global__ void __launch_bounds__(kCompactThreads)
 gather_rows_kernel(const __nv_bfloat16* __restrict__ hidden, int h, const int* __restrict__ idx,
-                   const int* __restrict__ count, long long cap, __nv_bfloat16* __restrict__ hidden_c) {
-  const long long kept = *count;
+                   const int* __restrict__ count, long long offset, long long rows,
+                   __nv_bfloat16* __restrict__ dst) {
+  long long kept = static_cast<long long>(*count) - offset;   // kept rows inside [offset, offset + rows)
+  kept = kept < 0 ? 0 : (kept > rows ? rows : kept);
   long long fill_to = (kept + 127) / 128 * 128;
-  if (fill_to > cap) fill_to = cap;
+  if (fill_to > rows) fill_to = rows;
   const int lane = threadIdx.x % kWarp;
   const long long warps = static_cast<long long>(gridDim.x) * (kCompactThreads / kWarp);
   const int vec_per_row = h / 8;  // 16-byte pieces
-  for (long long c = static_cast<long long>(blockIdx.x) * (kCompactThreads / kWarp) + threadIdx.x / kWarp; c < fill_to;
-       c += warps) {
-    uint4* dst = reinterpret_cast<uint4*>(hidden_c + c * h);
-    if (c < kept) {
-      const uint4* src = reinterpret_cast<const uint4*>(hidden + static_cast<long long>(idx[c]) * h);
-      for (int j = lane; j < vec_per_row; j += kWarp) dst[j] = __ldg(src + j);
+  for (long long r = static_cast<long long>(blockIdx.x) * (kCompactThreads / kWarp) + threadIdx.x / kWarp; r < fill_to;
+       r += warps) {
+    uint4* out = reinterpret_cast<uint4*>(dst + r * h);
+    if (r < kept) {
+      const uint4* src = reinterpret_cast<const uint4*>(hidden + static_cast<long long>(idx[offset + r]) * h);
+      for (int j = lane; j < vec_per_row; j += kWarp) out[j] = __ldg(src + j);
     } else {
-      for (int j = lane; j < vec_per_row; j += kWarp) dst[j] = make_uint4(0u, 0u, 0u, 0u);
+      for (int j = lane; j < vec_per_row; j += kWarp) out[j] = make_uint4(0u, 0u, 0u, 0u);
     }
   }
 }
@@ -210,8 +212,8 @@ bool compact_carve(void* ws, size_t ws_bytes, long long n, int h, bool backward,
   return true;
 }
 
-int compact_rows(const void* hidden, int h, const int32_t* targets, const uint8_t* row_mask, const float* g,
-                 const float* lse, long long n, const CompactBuffers& cb, cudaStream_t stream) {
+int compact_index(const int32_t* targets, const uint8_t* row_mask, const float* g, const float* lse, long long n,
+                  const CompactBuffers& cb, cudaStream_t stream) {
   long long rows_per_block = (n + kMaxCompactBlocks - 1) / kMaxCompactBlocks;
   rows_per_block = (rows_per_block + kCompactThreads - 1) / kCompactThreads * kCompactThreads;
   if (rows_per_block < kCompactThreads) rows_per_block = kCompactThreads;
@@ -225,14 +227,25 @@ int compact_rows(const void* hidden, int h, const int32_t* targets, const uint8_
   A3PO_LAUNCH(kKCompact, stream, (compact_fill_kernel<<<blocks, kCompactThreads, 0, stream>>>(
                                      row_mask, g, targets, lse, n, cb.cap, rows_per_block, cb.block_offsets, cb.count,
                                      cb.pos, cb.idx, cb.targets_c, cb.lse_c, cb.g_c)));
-  A3PO_RETURN_IF(after_launch());
+  return after_launch();
+}
+
+int gather_rows_range(const void* hidden, int h, const int* idx, const int* count, long long offset, long long rows,
+                      void* dst, cudaStream_t stream) {
+  if (rows <= 0) return A3PO_OK;
   int gather_blocks = sm_count() * 8;
-  const long long want = (cb.cap + 7) / 8;
+  const long long want = (rows + 7) / 8;
   if (gather_blocks > want) gather_blocks = static_cast<int>(want);
   A3PO_LAUNCH(kKCompact, stream, (gather_rows_kernel<<<gather_blocks, kCompactThreads, 0, stream>>>(
-                                     static_cast<const __nv_bfloat16*>(hidden), h, cb.idx, cb.count, cb.cap,
-                                     cb.hidden_c)));
+                                     static_cast<const __nv_bfloat16*>(hidden), h, idx, count, offset, rows,
+                                     static_cast<__nv_bfloat16*>(dst))));
   return after_launch();
+}
+
+int compact_rows(const void* hidden, int h, const int32_t* targets, const uint8_t* row_mask, const float* g,
+                 const float* lse, long long n, const CompactBuffers& cb, cudaStream_t stream) {
+  A3PO_RETURN_IF(compact_index(targets, row_mask, g, lse, n, cb, stream));
+  return gather_rows_range(hidden, h, cb.idx, cb.count, 0, cb.cap, cb.hidden_c, stream);
 }
 
 int scatter_rows(const void* src_c, int h, const int* pos, long long n, void* dst, cudaStream_t stream) {

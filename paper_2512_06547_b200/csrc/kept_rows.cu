@@ -55,7 +55,7 @@ target_logit_kernel(const __nv_bfloat16* __restrict__ hidden_c, const __nv_bfloa
   for (long long r = static_cast<long long>(blockIdx.x) * kWarpsPerBlock + threadIdx.x / kWarp; r < live; r += warps) {
     const long long c = offset + r;
     const int y = min(max(targets_c[c], 0), v - 1);
-    const uint4* a = reinterpret_cast<const uint4*>(hidden_c + c * h);
+    const uint4* a = reinterpret_cast<const uint4*>(hidden_c + r * h);   // hidden_c starts at the launch's first row
     const uint4* b = reinterpret_cast<const uint4*>(w + static_cast<long long>(y) * h);
     float acc = 0.f;
     for (int j = lane; j < vec; j += kWarp) acc = dot8(__ldg(a + j), __ldg(b + j), acc);
@@ -239,7 +239,7 @@ prepare_kept_backward_kernel(const int* __restrict__ count, long long offset, lo
         q[p * vpad + y] = __float2bfloat16_rn(-s);
         if (bwd_idx) bwd_idx[p] = static_cast<int>(t);
       }
-      const uint4* src = reinterpret_cast<const uint4*>(hidden_c ? hidden_c + c * h : hidden_batch + t * h);
+      const uint4* src = reinterpret_cast<const uint4*>(hidden_c ? hidden_c + (c - offset) * h : hidden_batch + t * h);
       for (int j = lane; j < vec; j += kWarp) {
         const uint4 in = __ldg(src + j);
         const __nv_bfloat162* x = reinterpret_cast<const __nv_bfloat162*>(&in);

@@ -41,6 +41,12 @@ bool compact_carve(void* ws, size_t ws_bytes, long long n, int h, bool backward,
 // Keeps row t iff (row_mask == null || row_mask[t] != 0) && (g == null || g[t] != 0).
 int compact_rows(const void* hidden, int h, const int32_t* targets, const uint8_t* row_mask, const float* g,
                  const float* lse, long long n, const CompactBuffers& cb, cudaStream_t stream);
+// The two halves of compact_rows: the index (count, pos, idx, compact scalars) for the whole batch, and the gather
+// of hidden rows for compact rows [offset, offset + rows) into dst (zero rows up to the next multiple of 128).
+int compact_index(const int32_t* targets, const uint8_t* row_mask, const float* g, const float* lse, long long n,
+                  const CompactBuffers& cb, cudaStream_t stream);
+int gather_rows_range(const void* hidden, int h, const int* idx, const int* count, long long offset, long long rows,
+                      void* dst, cudaStream_t stream);
 // dst[t, :] = src_c[pos[t], :] for kept rows, zero otherwise.
 int scatter_rows(const void* src_c, int h, const int* pos, long long n, void* dst, cudaStream_t stream);
 
@@ -70,9 +76,10 @@ size_t lmhead_tc_kept_bytes(long long rows, int v);
 int lmhead_fwd_keep_tc(const void* hidden, const void* w, const int32_t* targets, const float* zy, long long n, int h,
                        int v, float inv_t, int splits, float* part_s, float* part_e, void* q, const int* dyn_rows,
                        long long dyn_offset, uint32_t* status, cudaStream_t stream);
+// `select`: one device int of scratch (the tile choice made from the device-resident row count).
 int lmhead_grad_hidden_from_kept_tc(const void* q, const void* w, const float* row_scale, long long n, int h, int v,
-                                    void* grad_hidden, const int* dyn_rows, long long dyn_offset, uint32_t* status,
-                                    cudaStream_t stream);
+                                    void* grad_hidden, const int* dyn_rows, long long dyn_offset, int* select,
+                                    uint32_t* status, cudaStream_t stream);
 int lmhead_grad_w_from_kept_tc(const void* q, const void* hs, long long n, int h, int v, float* grad_w, int accumulate,
                                int zero_when_empty, const int* dyn_rows, long long dyn_offset, uint32_t* status,
                                cudaStream_t stream);
@@ -80,7 +87,8 @@ int lmhead_grad_w_from_kept_tc(const void* q, const void* hs, long long n, int h
 // Small per-row kernels around the kept-ratio path (kept_rows.cu).  `count` is the device-resident size of the
 // compact row space; every launch covers compact rows [offset, offset + rows) and arrays are indexed by compact row
 // unless they say otherwise.
-// zy[c] = dot(hidden_c[c, :], W[targets_c[c], :]) / T for the rows a GEMM launch may touch (up to the next 128).
+// hidden_c points at the launch's first row (row c of the compact space is hidden_c[c - offset, :]).
+// zy[c] = dot(hidden_c[c - offset, :], W[targets_c[c], :]) / T for the rows a GEMM launch may touch (up to the next 128).
 int target_logits(const void* hidden_c, const void* w, const int32_t* targets_c, const int* count, long long offset,
                   long long rows, int h, int v, float inv_t, float* zy, cudaStream_t stream);
 // s = sum of the split sums; lse = zy + log1p(s), logp = -log1p(s), sprime = s,

@@ -77,6 +77,10 @@ struct ItemMap {
   int zero_when_empty;   // dyn_is_k only: with no rows, store an all-zero output instead of doing nothing
   long long dyn_offset;
   long long dyn_cap;
+  // Optional device-side choice between two launches of the same contraction with different tiles: this launch
+  // does its work only if *select == select_value (the other one then exits at once).
+  const int* select;
+  int select_value;
 };
 
 struct Item {
@@ -528,6 +532,10 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   ItemMap im = im_static;
   int k_blocks = k_blocks_static;
   bool zero_output = false;  // K extent is empty: the product is the zero matrix
+  if (im.select != nullptr && *im.select != im.select_value) {
+    im.items = 0;
+    im.dyn_rows = nullptr;
+  }
   if (im.dyn_rows != nullptr) {
     long long rows = static_cast<long long>(*im.dyn_rows) - im.dyn_offset;
     rows = rows < 0 ? 0 : (rows > im.dyn_cap ? im.dyn_cap : rows);
@@ -814,6 +822,8 @@ struct DynRows {
   int zero_when_empty = 0;
   long long offset = 0;
   long long cap = 0;
+  const int* select = nullptr;
+  int select_value = 0;
 };
 
 // C[M, N] = sum_k A[m, k] B[n, k];  splits = 0 means one column tile per work item.
@@ -836,6 +846,8 @@ int launch_gemm(const Operand& a, const Operand& b, int splits, const typename E
   im.zero_when_empty = dyn.zero_when_empty;
   im.dyn_offset = dyn.offset;
   im.dyn_cap = dyn.cap;
+  im.select = dyn.select;
+  im.select_value = dyn.select_value;
   const int k_blocks = static_cast<int>((a.k_extent + BK - 1) / BK);
   auto kernel = gemm_tn_kernel<Epi, A_MN, B_MN, MT>;
   if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemBytes)) !=
@@ -851,19 +863,59 @@ int launch_gemm(const Operand& a, const Operand& b, int splits, const typename E
   return after_launch();
 }
 
-// The gradient contractions take the 256 x 256 tile (MT = 2); a tuning build can fall back to 128 x 256 for A/B runs.
+// Which tile a contraction over `rows` output rows and n_tiles column tiles should take.  The 256 x 256 tile moves a
+// third fewer operand bytes per flop, but its work items are twice as coarse; with few items per SM the idle tail
+// of the last wave costs more than that saves.  efficiency = items / (waves * SMs).
+__host__ __device__ inline int choose_mt(long long rows, int n_tiles, int sms) {
+  if (rows <= 0 || sms <= 0) return 2;
+  const long long i1 = (rows + BM - 1) / BM * n_tiles, i2 = (rows + 2 * BM - 1) / (2 * BM) * n_tiles;
+  const double e1 = static_cast<double>(i1) / static_cast<double>((i1 + sms - 1) / sms * sms);
+  const double e2 = static_cast<double>(i2) / static_cast<double>((i2 + sms - 1) / sms * sms);
+  return e2 >= 0.93 * e1 ? 2 : 1;
+}
+
+__global__ void choose_mt_kernel(const int* __restrict__ rows_ptr, long long offset, long long cap, int n_tiles,
+                                 int sms, int* __restrict__ out) {
+  long long rows = static_cast<long long>(*rows_ptr) - offset;
+  rows = rows < 0 ? 0 : (rows > cap ? cap : rows);
+  *out = choose_mt(rows, n_tiles, sms);
+}
+
+// The gradient contractions.  rows_are_m: the (possibly device-resident) row count is the M extent (grad_hidden),
+// so the tile is chosen from it, on the device when it lives there (both variants are launched, one of them
+// exits at once; `select` is a device int the choice is written to).  Otherwise (grad_w: M = V) the 256 x 256
+// tile always pays.
 template <class Epi, bool A_MN, bool B_MN>
-int launch_grad_gemm(const Operand& a, const Operand& b, const typename Epi::Params& ep, const DynRows& dyn,
-                     uint32_t* status, cudaStream_t stream) {
-  if (tuning_override("A3PO_GRAD_MT", 2) == 1) return launch_gemm<Epi, A_MN, B_MN, 1>(a, b, 0, ep, dyn, status, stream);
+int launch_grad_gemm(const Operand& a, const Operand& b, const typename Epi::Params& ep, DynRows dyn, bool rows_are_m,
+                     int* select, uint32_t* status, cudaStream_t stream) {
+  const int forced = tuning_override("A3PO_GRAD_MT", 0);
+  const int n_tiles = static_cast<int>((b.mn_extent + BN - 1) / BN);
+  int mt = 2;
+  if (forced == 1 || forced == 2) {
+    mt = forced;
+  } else if (rows_are_m && dyn.rows != nullptr && select != nullptr) {
+    A3PO_LAUNCH(kKCompact, stream, (choose_mt_kernel<<<1, 1, 0, stream>>>(dyn.rows, dyn.offset, dyn.cap, n_tiles,
+                                                                          sm_count(), select)));
+    A3PO_RETURN_IF(after_launch());
+    dyn.select = select;
+    dyn.select_value = 1;
+    A3PO_RETURN_IF((launch_gemm<Epi, A_MN, B_MN, 1>(a, b, 0, ep, dyn, status, stream)));
+    dyn.select_value = 2;
+    return launch_gemm<Epi, A_MN, B_MN, 2>(a, b, 0, ep, dyn, status, stream);
+  } else if (rows_are_m) {
+    mt = choose_mt(a.mn_extent, n_tiles, sm_count());
+  }
+  if (mt == 1) return launch_gemm<Epi, A_MN, B_MN, 1>(a, b, 0, ep, dyn, status, stream);
   return launch_gemm<Epi, A_MN, B_MN, 2>(a, b, 0, ep, dyn, status, stream);
 }
 
 // Scratch of the backward: one bf16 dz chunk [chunk_rows, vpad].
-size_t bwd_ws_layout(long long chunk_rows, int v) {
+size_t bwd_dz_bytes(long long chunk_rows, int v) {
   const size_t vpad = round_up(static_cast<size_t>(v), 8);
   return round_up(static_cast<size_t>(chunk_rows) * vpad * 2, 256);
 }
+// ... followed by one int (the tile choice of the chunk's grad_hidden launch)
+size_t bwd_ws_layout(long long chunk_rows, int v) { return bwd_dz_bytes(chunk_rows, v) + 256; }
 
 }  // namespace
 
@@ -980,6 +1032,7 @@ int lmhead_bwd_tc(const void* hidden_, const void* w_, const int32_t* targets, c
   __nv_bfloat16* grad_hidden = static_cast<__nv_bfloat16*>(grad_hidden_);
   if (bwd_ws_layout(chunk_rows, v) > ws_bytes) return A3PO_ERR_WORKSPACE;
   __nv_bfloat16* dz = static_cast<__nv_bfloat16*>(ws);  // [chunk_rows, vpad]
+  int* select = reinterpret_cast<int*>(static_cast<char*>(ws) + bwd_dz_bytes(chunk_rows, v));
   const int vpad = static_cast<int>(round_up(static_cast<size_t>(v), 8));
 
   for (long long r0 = 0; r0 < n; r0 += chunk_rows) {
@@ -1000,11 +1053,11 @@ int lmhead_bwd_tc(const void* hidden_, const void* w_, const int32_t* targets, c
     // grad_hidden[t, j] = sum_v dz[t, v] W[v, j]:  A = dz (K = v contiguous), B = W read N-major
     StoreBf16Epilogue::Params hp{grad_hidden + r0 * h, h, nc, h, nullptr};
     A3PO_RETURN_IF((launch_grad_gemm<StoreBf16Epilogue, false, true>(Operand{dz, nc, v, vpad}, Operand{w, h, v, h}, hp,
-                                                                     dyn_m, status, stream)));
+                                                                     dyn_m, true, select, status, stream)));
     // grad_w[v, j] (+)= sum_t dz[t, v] hidden[t, j]:  A = dz read M-major, B = hidden read N-major (K = t)
     StoreF32Epilogue::Params wp{grad_w, h, v, h, (accumulate || r0 > 0) ? 1 : 0};
     A3PO_RETURN_IF((launch_grad_gemm<StoreF32Epilogue, true, true>(Operand{dz, v, nc, vpad}, Operand{hid_c, h, nc, h},
-                                                                   wp, dyn_k, status, stream)));
+                                                                   wp, dyn_k, false, nullptr, status, stream)));
   }
   return A3PO_OK;
 }
@@ -1015,8 +1068,8 @@ int lmhead_bwd_tc(const void* hidden_, const void* w_, const int32_t* targets, c
 //   grad_w[v, :]    (+)= sum_r q[r, v] hs[r, :]                 hs = row_scale * hidden, made by the caller
 // which equal dz W and dz^T hidden for dz[r, v] = row_scale[r] q[r, v].
 int lmhead_grad_hidden_from_kept_tc(const void* q_, const void* w_, const float* row_scale, long long n, int h, int v,
-                                    void* grad_hidden_, const int* dyn_rows, long long dyn_offset, uint32_t* status,
-                                    cudaStream_t stream) {
+                                    void* grad_hidden_, const int* dyn_rows, long long dyn_offset, int* select,
+                                    uint32_t* status, cudaStream_t stream) {
   const __nv_bfloat16* q = static_cast<const __nv_bfloat16*>(q_);
   const __nv_bfloat16* w = static_cast<const __nv_bfloat16*>(w_);
   const int vpad = static_cast<int>(round_up(static_cast<size_t>(v), 8));
@@ -1025,8 +1078,8 @@ int lmhead_grad_hidden_from_kept_tc(const void* q_, const void* w_, const float*
   dyn_m.offset = dyn_offset;
   dyn_m.cap = n;
   StoreBf16Epilogue::Params hp{static_cast<__nv_bfloat16*>(grad_hidden_), h, n, h, row_scale};
-  return launch_grad_gemm<StoreBf16Epilogue, false, true>(Operand{q, n, v, vpad}, Operand{w, h, v, h}, hp, dyn_m,
-                                                          status, stream);
+  return launch_grad_gemm<StoreBf16Epilogue, false, true>(Operand{q, n, v, vpad}, Operand{w, h, v, h}, hp, dyn_m, true,
+                                                          select, status, stream);
 }
 
 int lmhead_grad_w_from_kept_tc(const void* q_, const void* hs_, long long n, int h, int v, float* grad_w,
@@ -1042,8 +1095,8 @@ int lmhead_grad_w_from_kept_tc(const void* q_, const void* hs_, long long n, int
   dyn_k.is_k = 1;
   dyn_k.zero_when_empty = zero_when_empty;
   StoreF32Epilogue::Params wp{grad_w, h, v, h, accumulate ? 1 : 0};
-  return launch_grad_gemm<StoreF32Epilogue, true, true>(Operand{q, v, n, vpad}, Operand{hs, h, n, h}, wp, dyn_k,
-                                                        status, stream);
+  return launch_grad_gemm<StoreF32Epilogue, true, true>(Operand{q, v, n, vpad}, Operand{hs, h, n, h}, wp, dyn_k, false,
+                                                        nullptr, status, stream);
 }
 
 }  // namespace a3po

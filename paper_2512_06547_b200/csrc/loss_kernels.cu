@@ -157,7 +157,11 @@ __device__ __forceinline__ void finalize_block(const LossPartial* partials, int 
                                                a3po_stats* stats, LossPartial* sh /*[kLossThreads]*/) {
   LossPartial mine{0.0, 0, 0, 0.f, 3.4e38f};
   for (int i = threadIdx.x; i < count; i += kLossThreads) {
-    const LossPartial q = partials[i];
+    const uint4 lo = __ldcg(reinterpret_cast<const uint4*>(partials + i));       // written by other blocks
+    const uint4 hi = __ldcg(reinterpret_cast<const uint4*>(partials + i) + 1);
+    LossPartial q;
+    memcpy(&q, &lo, 16);
+    memcpy(reinterpret_cast<char*>(&q) + 16, &hi, 16);
     mine.sum += q.sum;
     mine.n_valid += q.n_valid;
     mine.n_clipped += q.n_clipped;
@@ -190,7 +194,11 @@ __device__ __forceinline__ void finalize_block(const LossPartial* partials, int 
 }
 
 // This block's share of M = number of non-zero mask bytes (16 mask bytes per load where alignment
-// allows); the block total goes to block_counts[blockIdx.x].
+// allows, four loads in flight per thread); the block total goes to block_counts[blockIdx.x].
+__device__ __forceinline__ int popc16(const uint4 m) {
+  return (__popc(__vcmpne4(m.x, 0u)) + __popc(__vcmpne4(m.y, 0u)) + __popc(__vcmpne4(m.z, 0u)) +
+          __popc(__vcmpne4(m.w, 0u))) >> 3;
+}
 __device__ __forceinline__ void count_mask_block(const uint8_t* mask, long long n, long long* block_counts,
                                                  long long* sh /*[kLossThreads / kWarp]*/) {
   long long count = 0;
@@ -200,11 +208,14 @@ __device__ __forceinline__ void count_mask_block(const uint8_t* mask, long long 
   long long done = 0;
   if (vec) {
     const long long groups = n >> 4;
-    for (long long g = tid; g < groups; g += nthreads) {
-      const uint4 m = __ldg(reinterpret_cast<const uint4*>(mask) + g);
-      count += (__popc(__vcmpne4(m.x, 0u)) + __popc(__vcmpne4(m.y, 0u)) +
-                __popc(__vcmpne4(m.z, 0u)) + __popc(__vcmpne4(m.w, 0u))) >> 3;
+    const uint4* m16 = reinterpret_cast<const uint4*>(mask);
+    long long g = tid;
+    for (; g + 3 * nthreads < groups; g += 4 * nthreads) {
+      const uint4 a = __ldg(m16 + g), b = __ldg(m16 + g + nthreads), c = __ldg(m16 + g + 2 * nthreads),
+                  d = __ldg(m16 + g + 3 * nthreads);
+      count += popc16(a) + popc16(b) + popc16(c) + popc16(d);
     }
+    for (; g < groups; g += nthreads) count += popc16(__ldg(m16 + g));
     done = groups << 4;
   }
   for (long long t = done + tid; t < n; t += nthreads) count += mask[t] != 0;
@@ -222,7 +233,7 @@ __device__ __forceinline__ void count_mask_block(const uint8_t* mask, long long 
 __device__ __forceinline__ void sum_counts_block(const long long* block_counts, int count, long long* out,
                                                  long long* sh /*[kLossThreads]*/) {
   long long mine = 0;
-  for (int i = threadIdx.x; i < count; i += kLossThreads) mine += block_counts[i];
+  for (int i = threadIdx.x; i < count; i += kLossThreads) mine += __ldcg(block_counts + i);  // written by other blocks
   sh[threadIdx.x] = mine;
   __syncthreads();
   for (int s = kLossThreads / 2; s > 0; s >>= 1) {
@@ -238,16 +249,20 @@ template <int MODE, bool VEC, bool EXPLICIT>
 __global__ void __launch_bounds__(kLossThreads, kBlocksPerSm) loss_kernel(LossArgs p, LossPartial* partials,
                                                                           LossPhases ph) {
   __shared__ LossPartial sh[kLossThreads];
+  __shared__ long long s_m;
   if (ph.bits & kPhaseCountMask) {
+    // every block counts its share, then (one grid-wide barrier later) adds up all the shares itself, in index
+    // order: the same M in every block without a second barrier
     long long* shc = reinterpret_cast<long long*>(sh);
     count_mask_block(p.mask, p.n, ph.block_counts, shc);
     cg::this_grid().sync();
-    if (blockIdx.x == 0) sum_counts_block(ph.block_counts, gridDim.x, ph.n_valid, shc);
-    cg::this_grid().sync();
+    sum_counts_block(ph.block_counts, gridDim.x, &s_m, shc);
+    __syncthreads();
+    if (blockIdx.x == 0 && threadIdx.x == 0) *ph.n_valid = s_m;
   }
   float coef = 0.f;
   if (MODE != kFwd) {
-    long long m = *reinterpret_cast<const volatile long long*>(p.n_valid_ptr);
+    long long m = (ph.bits & kPhaseCountMask) ? s_m : *p.n_valid_ptr;
     float gl = p.grad_loss ? *p.grad_loss : 1.0f;
     coef = (m > 0) ? -gl / static_cast<float>(m) : 0.f;
   }

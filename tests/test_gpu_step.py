@@ -157,7 +157,7 @@ def test_keeping_step_in_several_row_chunks():
     dt = a3po.A3PO_BF16
     big = a3po.a3po_train_step_workspace_bytes(wl.N, wl.H, wl.V, dt)
     vpad = (wl.V + 7) // 8 * 8
-    per_row = 2 * vpad + 4 * wl.H + 2 * 4 * 64 + 5 * 4          # kept ratios, hs, ghc, split sums, row plan
+    per_row = 2 * vpad + 6 * wl.H + 2 * 4 * 64 + 5 * 4          # kept ratios, hidden_c + hs + ghc, split sums, row plan
     cap = (wl.N + 127) // 128 * 128
     assert cap >= 3 * 2048
     part = big - (cap - 2048 - 512) * per_row                    # room for chunks of a bit over 2048 rows
