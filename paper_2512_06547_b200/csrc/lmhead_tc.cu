@@ -24,6 +24,7 @@
 // Every mbarrier wait is bounded; on expiry the CTA raises A3PO_STATUS_WAIT_TIMEOUT in the
 // caller's status word, releases its TMEM and exits.
 
+#include <cstdio>
 #include <cstdlib>
 #include <cstring>
 #include <mutex>
@@ -775,6 +776,187 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #endif
 }
 
+// ------------------------------------------------------------------------------------ the pair kernel
+// The same contraction with both operands K-major, run by pairs of CTAs on neighbouring SMs (clusters of two,
+// tcgen05 cta_group::2).  A pair owns a 256-row output tile: each CTA loads its own 128 rows of A and only ITS
+// half (128 of 256 rows) of every B tile, the leader's MMAs (M = 256) read both halves, and each CTA finds its
+// 128 x 256 accumulator in its own tensor memory and runs the epilogue on it.  Per flop a CTA then pulls a third
+// fewer operand bytes out of L2 and through shared memory than with a full B tile of its own, which is where the
+// single-CTA kernel saturates when the SM clock is high.  Accumulators stay double-buffered (the epilogue of one
+// tile overlaps the MMAs of the next), so this is the kernel for the epilogue-heavy forward contractions.
+// Every CTA fetches its own tiles (no multicast).  Barriers: "stage filled" lives in the leader (both CTAs' loads
+// signal it), "stage free" and "accumulator ready" exist in both CTAs (the leader's commit arrives on both),
+// "accumulator free" lives in the leader and collects the eight epilogue warps of the pair.
+constexpr int kPairStages = 6;
+constexpr uint32_t kPairStageBytes = kABytes + kBBytes / 2;   // per CTA: 128 x 64 of A, 128 x 64 of B
+constexpr size_t kPairSmemBytes = 1024 + kPairStages * kPairStageBytes + 2 * kSlabBytes + 256;
+
+template <class Epi>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kTcThreads, 1)
+gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                 const __grid_constant__ CUtensorMap map_c, ItemMap im_static, int k_blocks,
+                 typename Epi::Params ep, uint32_t* status) {
+  constexpr int kPairRows = 2 * BM;
+  ItemMap im = im_static;   // m_tiles counts 256-row pair tiles here
+  if (im.dyn_rows != nullptr) {
+    long long rows = static_cast<long long>(*im.dyn_rows) - im.dyn_offset;
+    rows = rows < 0 ? 0 : (rows > im.dyn_cap ? im.dyn_cap : rows);
+    im.m_tiles = static_cast<int>((rows + kPairRows - 1) / kPairRows);
+    im.items = static_cast<long long>(im.m_tiles) * im.splits;
+  }
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* smem_a = smem;
+  uint8_t* smem_b = smem + kPairStages * kABytes;
+  uint8_t* smem_slabs = smem + kPairStages * kPairStageBytes;
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem_slabs + 2 * kSlabBytes);
+  uint64_t* empty_bar = full_bar + kPairStages;
+  uint64_t* tmem_full_bar = empty_bar + kPairStages;
+  uint64_t* tmem_empty_bar = tmem_full_bar + 2;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tmem_empty_bar + 2);
+  volatile uint32_t* abort_flag = tmem_slot + 1;
+
+  const int warp = threadIdx.x / kWarp;
+  const int lane = threadIdx.x % kWarp;
+  const uint32_t rank = cluster_ctarank();         // 0 = leader
+  const long long pair_id = blockIdx.x >> 1;
+  const long long n_pairs = gridDim.x >> 1;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < kPairStages; ++i) {
+      mbar_init(&full_bar[i], 1);    // used in the leader only: its producer's arrive + the bytes of both CTAs
+      mbar_init(&empty_bar[i], 1);   // one arrival: the leader's commit
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&tmem_full_bar[i], 1);
+      mbar_init(&tmem_empty_bar[i], 8);  // used in the leader only: four epilogue warps in each CTA
+    }
+    *abort_flag = 0;
+    fence_mbar_init();
+  }
+  if (warp == 0 && lane == 0) {
+    prefetch_tensormap(&map_a);
+    prefetch_tensormap(&map_b);
+  }
+  if (warp == 1) {   // the same warp in both CTAs, together
+    tmem_alloc_pair(tmem_slot, kTmemCols);
+    tmem_relinquish_alloc_permit_pair();
+  }
+  tcgen05_fence_before_sync();
+  __syncthreads();
+  cluster_sync_all();   // the peer's barriers exist before anything signals them
+  tcgen05_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  bool ok = true;
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer (both CTAs)
+    if (elect_one()) {
+      const uint32_t leader_full = map_to_cta(smem_u32(&full_bar[0]), 0);
+      int stage = 0;
+      uint32_t phase = 0;
+      for (long long i = pair_id; i < im.items && ok; i += n_pairs) {
+        const Item it = decode_item(im, i);
+        const int row0 = it.m_tile * kPairRows + static_cast<int>(rank) * BM;
+        for (int nt = it.n_begin; nt < it.n_end && ok; ++nt) {
+          const int col0 = nt * BN + static_cast<int>(rank) * (BN / 2);
+          for (int kb = 0; kb < k_blocks; ++kb) {
+            if (!mbar_wait(&empty_bar[stage], phase ^ 1u, abort_flag)) { ok = false; break; }
+            if (rank == 0) mbar_arrive_expect_tx(&full_bar[stage], 2 * kPairStageBytes);
+            const uint32_t bar = leader_full + static_cast<uint32_t>(stage * sizeof(uint64_t));
+            tma_load_2d_pair(smem_a + stage * kABytes, &map_a, bar, kb * BK, row0);
+            tma_load_2d_pair(smem_b + stage * (kBBytes / 2), &map_b, bar, kb * BK, col0);
+            if (++stage == kPairStages) { stage = 0; phase ^= 1u; }
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer (leader only)
+    if (rank == 0 && elect_one()) {
+      constexpr uint32_t idesc = umma_idesc_bf16_f32(kPairRows, BN, false, false);
+      int stage = 0;
+      uint32_t phase = 0;
+      int acc = 0;
+      uint32_t acc_phase = 0;
+      for (long long i = pair_id; i < im.items && ok; i += n_pairs) {
+        const Item it = decode_item(im, i);
+        for (int nt = it.n_begin; nt < it.n_end && ok; ++nt) {
+          if (!mbar_wait(&tmem_empty_bar[acc], acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+          tcgen05_fence_after_sync();
+          const uint32_t tmem_d = tmem_base + static_cast<uint32_t>(acc * BN);
+          for (int kb = 0; kb < k_blocks; ++kb) {
+            if (!mbar_wait(&full_bar[stage], phase, abort_flag)) { ok = false; break; }
+            tcgen05_fence_after_sync();
+            const uint64_t desc_a = umma_desc_k_major_sw128(smem_u32(smem_a + stage * kABytes));
+            const uint64_t desc_b = umma_desc_k_major_sw128(smem_u32(smem_b + stage * (kBBytes / 2)));
+#pragma unroll
+            for (int k = 0; k < BK / 16; ++k)
+              umma_bf16_pair(tmem_d, desc_a + 2 * k, desc_b + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+            umma_commit_pair(&empty_bar[stage], 3);   // both CTAs may refill the stage
+            if (++stage == kPairStages) { stage = 0; phase ^= 1u; }
+          }
+          if (ok) umma_commit_pair(&tmem_full_bar[acc], 3);
+          if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue warps (both CTAs)
+    const int quarter = warp & 3;
+    const int row_in_tile = quarter * 32 + lane;
+    const uint32_t leader_tmem_empty = map_to_cta(smem_u32(&tmem_empty_bar[0]), 0);
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    Epi epi;
+    SlabStore st;
+    st.slab0 = smem_slabs;
+    st.slab1 = smem_slabs + kSlabBytes;
+    st.map = &map_c;
+    st.row_in_tile = row_in_tile;
+    st.issuer = (threadIdx.x == 2 * kWarp);
+    for (long long i = pair_id; i < im.items && ok; i += n_pairs) {
+      const Item it = decode_item(im, i);
+      const int tile_row0 = it.m_tile * kPairRows + static_cast<int>(rank) * BM;
+      epi.begin(ep, static_cast<long long>(tile_row0) + row_in_tile);
+      for (int nt = it.n_begin; nt < it.n_end && ok; ++nt) {
+        ok = all_epilogue_threads(mbar_wait(&tmem_full_bar[acc], acc_phase, abort_flag));
+        if (!ok) break;
+        tcgen05_fence_after_sync();
+        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(acc * BN);
+#pragma unroll 1
+        for (int c = 0; c < BN / kEpiChunk; ++c) {
+          uint32_t r[kEpiChunk];
+          tmem_ld_32x32(taddr + static_cast<uint32_t>(c * kEpiChunk), r);
+          tmem_ld_wait();
+          epi.chunk(ep, tile_row0, nt * BN + c * kEpiChunk, r, st);
+        }
+        tcgen05_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(leader_tmem_empty + static_cast<uint32_t>(acc * sizeof(uint64_t)));
+        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      }
+      if (ok) epi.end(ep, static_cast<long long>(tile_row0) + row_in_tile, it.split);
+    }
+    st.drain();
+  }
+
+  if (!ok) {
+    *abort_flag = 1;
+    if (status) atomicOr(status, A3PO_STATUS_WAIT_TIMEOUT);
+    __nanosleep(200000);
+  }
+  // neither CTA may leave (or give up its tensor memory) while the other can still read its shared memory or
+  // signal its barriers
+  tcgen05_fence_before_sync();
+  __syncthreads();
+  cluster_sync_all();
+  if (warp == 1) {
+    tcgen05_fence_after_sync();
+    tmem_dealloc_pair(tmem_base, kTmemCols);
+  }
+}
+
 // ------------------------------------------------------------------------------------ host side
 // One GEMM operand as it lies in memory (bf16, row-major with `pitch` elements per row).
 //   K-major : tensor [mn_extent rows, k_extent cols]   -> boxes of tile_mn rows x 64 k
@@ -859,6 +1041,81 @@ int launch_gemm(const Operand& a, const Operand& b, int splits, const typename E
   if (grid > im.items) grid = im.items;
   if (grid < 1) return A3PO_OK;
   A3PO_LAUNCH(Epi::kKernelId, stream, (kernel<<<static_cast<unsigned>(grid), kTcThreads, kSmemBytes, stream>>>(
+                                          map_a, map_b, map_c, im, k_blocks, ep, status)));
+  return after_launch();
+}
+
+// Pairs of CTAs that can be resident at once (the kernel is persistent: one pair per two SMs).
+template <class Epi>
+int pair_capacity() {
+  static std::mutex mu;
+  static int cached[64];
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
+    cudaGetLastError();
+    return 0;
+  }
+  std::lock_guard<std::mutex> lock(mu);
+  if (cached[dev] == 0) {
+    auto kernel = gemm_pair_kernel<Epi>;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kPairSmemBytes)) !=
+        cudaSuccess) {
+      cudaGetLastError();
+      return 0;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(sm_count() / 2 * 2));
+    cfg.blockDim = dim3(kTcThreads);
+    cfg.dynamicSmemBytes = kPairSmemBytes;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 2;
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    int clusters = 0;
+    if (cudaOccupancyMaxActiveClusters(&clusters, kernel, &cfg) != cudaSuccess) {
+      cudaGetLastError();
+      clusters = -1;
+    }
+    cached[dev] = clusters > 0 ? clusters : -1;
+#ifdef A3PO_TUNING
+    fprintf(stderr, "[a3po tuning] CTA pairs resident at once: %d\n", clusters);
+#endif
+  }
+  return cached[dev] > 0 ? cached[dev] : 0;
+}
+
+// C[M, N] = sum_k A[m, k] B[n, k], both K-major, on CTA pairs; `splits` vocabulary splits per 256-row pair tile.
+template <class Epi>
+int launch_pair_gemm(const Operand& a, const Operand& b, int splits, const typename Epi::Params& ep, const DynRows& dyn,
+                     uint32_t* status, cudaStream_t stream) {
+  const int pairs_max = pair_capacity<Epi>();
+  if (pairs_max <= 0) return A3PO_ERR_UNSUPPORTED;
+  CUtensorMap map_a, map_b, map_c;
+  A3PO_RETURN_IF(make_map(&map_a, a, false, BM));
+  A3PO_RETURN_IF(make_map(&map_b, b, false, BN / 2));
+  A3PO_RETURN_IF(Epi::make_c_map(ep, &map_c));
+  ItemMap im;
+  im.m_tiles = static_cast<int>((a.mn_extent + 2 * BM - 1) / (2 * BM));
+  im.n_tiles = static_cast<int>((b.mn_extent + BN - 1) / BN);
+  im.splits = splits > 0 ? splits : im.n_tiles;
+  im.items = static_cast<long long>(im.m_tiles) * im.splits;
+  im.group_m = tuning_override("A3PO_GROUP_M", kGroupM / 2);
+  im.dyn_rows = dyn.rows;
+  im.dyn_is_k = 0;
+  im.zero_when_empty = 0;
+  im.dyn_offset = dyn.offset;
+  im.dyn_cap = dyn.cap;
+  im.select = nullptr;
+  im.select_value = 0;
+  const int k_blocks = static_cast<int>((a.k_extent + BK - 1) / BK);
+  long long pairs = pairs_max;
+  if (pairs > im.items) pairs = im.items;
+  if (pairs < 1) return A3PO_OK;
+  auto kernel = gemm_pair_kernel<Epi>;
+  A3PO_LAUNCH(Epi::kKernelId, stream, (kernel<<<static_cast<unsigned>(2 * pairs), kTcThreads, kPairSmemBytes, stream>>>(
                                           map_a, map_b, map_c, im, k_blocks, ep, status)));
   return after_launch();
 }
@@ -954,14 +1211,26 @@ bool lmhead_tc_supported(const void* hidden, const void* w, long long n, int h, 
          n < (1ll << 31) - 256;
 }
 
+// Whether the forward contractions run on CTA pairs (gemm_pair_kernel).  Off: measured on B200 under its power
+// cap (seconds-long loops on one GPU) the pair kernel sustains 1083 TFLOP/s against 1241 for the single-CTA
+// kernel on the same forward, although its tensor pipe is busier when the clock is free (99 % against 90 % under
+// the profiler).  A tuning build switches it on with A3PO_FWD_PAIR=1 for comparisons and for its parity test.
+bool fwd_uses_pairs() {
+  if (tuning_override("A3PO_FWD_PAIR", 2) != 1) return false;
+  return pair_capacity<KeepEpilogue<false>>() > 0;
+}
+
 // Picks the number of vocabulary splits so that (row tiles x splits) items spread evenly over
-// the SMs (static round-robin) while every item still sweeps several column tiles.
+// the workers (SMs, or CTA pairs with 256-row tiles; static round-robin) while every item still sweeps several
+// column tiles.
 int lmhead_tc_fwd_splits(long long n, int v) {
-  const long long m_tiles = (n + BM - 1) / BM;
+  const bool pairs = fwd_uses_pairs();
+  const int tile_rows = pairs ? 2 * BM : BM;
+  const long long m_tiles = (n + tile_rows - 1) / tile_rows;
   const int n_tiles = (v + BN - 1) / BN;
   if (m_tiles <= 0) return 1;
-  int sms = sm_count();
-  if (sms <= 0) sms = 148;
+  int workers = pairs ? pair_capacity<KeepEpilogue<false>>() : sm_count();
+  if (workers <= 0) workers = pairs ? 74 : 148;
   const int forced = tuning_override("A3PO_FWD_SPLITS", 0);
   if (forced > 0) return forced < n_tiles ? (forced < 64 ? forced : 64) : n_tiles;
   const int s_max = n_tiles < 64 ? n_tiles : 64;
@@ -970,7 +1239,7 @@ int lmhead_tc_fwd_splits(long long n, int v) {
   double best_cost = 1e300;
   for (int s = s_min; s <= s_max; ++s) {
     const long long items = m_tiles * s;
-    const long long waves = (items + sms - 1) / sms;
+    const long long waves = (items + workers - 1) / workers;
     const long long tiles_per_item = (n_tiles + s - 1) / s;
     const double cost = static_cast<double>(waves) * (static_cast<double>(tiles_per_item) + 0.5);
     if (cost < best_cost - 1e-9) { best_cost = cost; best = s; }
@@ -986,11 +1255,14 @@ int lmhead_fwd_tc(const void* hidden, const void* w, const int32_t* targets, lon
   DynRows dyn;
   dyn.rows = dyn_rows;
   dyn.cap = n;
+  const bool pairs = fwd_uses_pairs();
   if (part_ent) {
     FwdEpilogue<true>::Params p{targets, n, v, inv_t * kLog2e, inv_t, part, part_ent, zy};
+    if (pairs) return launch_pair_gemm<FwdEpilogue<true>>(a, b, splits, p, dyn, status, stream);
     return launch_gemm<FwdEpilogue<true>, false, false>(a, b, splits, p, dyn, status, stream);
   }
   FwdEpilogue<false>::Params p{targets, n, v, inv_t * kLog2e, inv_t, part, nullptr, zy};
+  if (pairs) return launch_pair_gemm<FwdEpilogue<false>>(a, b, splits, p, dyn, status, stream);
   return launch_gemm<FwdEpilogue<false>, false, false>(a, b, splits, p, dyn, status, stream);
 }
 
@@ -1009,13 +1281,16 @@ int lmhead_fwd_keep_tc(const void* hidden, const void* w, const int32_t* targets
   dyn.offset = dyn_offset;
   dyn.cap = n;
   const int vpad = static_cast<int>(round_up(static_cast<size_t>(v), 8));
+  const bool pairs = fwd_uses_pairs();
   if (part_e) {
     KeepEpilogue<true>::Params p{targets, zy, n, v, vpad, inv_t * kLog2e, inv_t, part_s, part_e,
                                  static_cast<__nv_bfloat16*>(q)};
+    if (pairs) return launch_pair_gemm<KeepEpilogue<true>>(a, b, splits, p, dyn, status, stream);
     return launch_gemm<KeepEpilogue<true>, false, false>(a, b, splits, p, dyn, status, stream);
   }
   KeepEpilogue<false>::Params p{targets, zy, n, v, vpad, inv_t * kLog2e, inv_t, part_s, nullptr,
                                 static_cast<__nv_bfloat16*>(q)};
+  if (pairs) return launch_pair_gemm<KeepEpilogue<false>>(a, b, splits, p, dyn, status, stream);
   return launch_gemm<KeepEpilogue<false>, false, false>(a, b, splits, p, dyn, status, stream);
 }
 
