@@ -240,6 +240,27 @@ int a3po_decoupled_loss_fwd_bwd(const float* logp, const float* behav_logp, cons
                                 size_t ws_bytes, void* stream);
 
 /* --------------------------------------------------------------------------------------------
+ * Helpers for data-parallel training over sequences (no counterpart in the paper, which states E_t
+ * of Eq. 2 for one batch).  The path is per token except the masked mean, so a job that shards its
+ * sequences over ranks gets the whole-job loss and gradients from per-rank calls as
+ *     L = sum_r (M_r / M) L_r,     grad = sum_r (M_r / M) grad_r,      M = sum_r M_r,
+ * where L_r, grad_r are what rank r computes with its local mean.  a3po_mask_count gives M_r before
+ * the step (the mask is an input), the caller all-reduces it, a3po_dp_loss_scale turns the two
+ * counts into the weight M_r / M, and a3po_train_step takes that weight as `loss_scale`, so its
+ * gradients come out already weighted and one sum all-reduce of grad_w (and of the weighted loss)
+ * finishes the job; grad_hidden and grad_logp stay local.
+ *
+ * a3po_mask_count: *count (int64, device) = number of non-zero mask bytes; ws of
+ *   a3po_mask_count_workspace_bytes() bytes.
+ * a3po_dp_loss_scale: *scale = M_local / M_global (0 if M_global == 0), all device scalars; when
+ *   loss_local is given, *weighted_loss = *scale * *loss_local as well.
+ * ------------------------------------------------------------------------------------------ */
+size_t a3po_mask_count_workspace_bytes(void);
+int a3po_mask_count(const uint8_t* mask, int64_t N, int64_t* count, void* ws, size_t ws_bytes, void* stream);
+int a3po_dp_loss_scale(const int64_t* m_local, const int64_t* m_global, const float* loss_local,
+                       float* scale, float* weighted_loss, void* stream);
+
+/* --------------------------------------------------------------------------------------------
  * GRPO advantages (Sec. 4.1: "estimate advantages using group reward normalization"; the paper
  * gives no formula, the customary one is used).  Sequences come in consecutive groups of
  * `group_size` responses to the same prompt:
@@ -314,7 +335,9 @@ int a3po_loss_fwd_static(const float* logp, const float* behav_logp, const int32
  * chunks) plus a gathered copy of hidden.  With a smaller workspace (at least
  * a3po_train_step_min_workspace_bytes) or fp32 inputs the three calls are made as they are.
  * logp, lse, grad_logp: fp32 [N] outputs.  entropy: fp32 [N] or NULL (policy entropy per row,
- * Fig. 4).  Other arguments as in the individual calls.
+ * Fig. 4).  loss_scale: fp32 device scalar or NULL (= 1): every gradient (grad_logp, grad_hidden,
+ * grad_w) is multiplied by it, the reported loss is not; data-parallel callers pass M_local /
+ * M_global (see a3po_dp_loss_scale).  Other arguments as in the individual calls.
  * ------------------------------------------------------------------------------------------ */
 size_t a3po_train_step_min_workspace_bytes(int64_t N, int H, int V, a3po_dtype dt);
 size_t a3po_train_step_workspace_bytes(int64_t N, int H, int V, a3po_dtype dt);
@@ -324,8 +347,8 @@ int a3po_train_step(const void* hidden, const int32_t* targets, const float* beh
                     int V, a3po_dtype dt, int32_t current_version, float clip_eps,
                     float inv_temperature, const void* w, float* grad_w, int accumulate_grad_w,
                     void* grad_hidden, float* logp, float* lse, float* entropy, float* grad_logp,
-                    float* loss, a3po_stats* stats, void* ws, size_t ws_bytes, uint32_t* status,
-                    void* stream);
+                    float* loss, a3po_stats* stats, const float* loss_scale, void* ws, size_t ws_bytes,
+                    uint32_t* status, void* stream);
 
 /* --------------------------------------------------------------------------------------------
  * The same pass with per-step inputs in HOST memory (no counterpart in the paper; this is the

@@ -75,7 +75,11 @@ _SIGNATURES = {
     "a3po_train_step_min_workspace_bytes": (c_size_t, [c_int64, c_int, c_int, c_int]),
     "a3po_train_step": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_int, c_int, c_int,
                                 c_int32, c_float, c_float, c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_void_p,
-                                c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p, c_void_p]),
+                                c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p,
+                                c_void_p]),
+    "a3po_mask_count_workspace_bytes": (c_size_t, []),
+    "a3po_mask_count": (c_int, [c_void_p, c_int64, c_void_p, c_void_p, c_size_t, c_void_p]),
+    "a3po_dp_loss_scale": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
     "a3po_train_step_host": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_int, c_int,
                                      c_int, c_int32, c_float, c_float, c_void_p, c_void_p, c_int, c_void_p, c_void_p,
                                      c_size_t, c_void_p, c_size_t, c_void_p, c_void_p, c_void_p, c_void_p]),
@@ -392,8 +396,8 @@ def a3po_train_step_min_workspace_bytes(N, H, V, dt) -> int:
 
 
 def a3po_train_step(hidden, w, targets, behav_logp, versions, current_version, adv, mask, clip_eps, logp, lse,
-                    grad_logp, loss, grad_hidden, grad_w, ws, *, stats=None, entropy=None, accumulate_grad_w=False,
-                    inv_temperature=1.0, status=None, stream=None):
+                    grad_logp, loss, grad_hidden, grad_w, ws, *, stats=None, entropy=None, loss_scale=None,
+                    accumulate_grad_w=False, inv_temperature=1.0, status=None, stream=None):
     """token_logprobs_fwd -> loss_fwd_bwd -> token_logprobs_bwd in one call; with the recommended workspace the
     backward reuses the softmax kept by the forward instead of recomputing the logits."""
     dt = _dtype_code(hidden)
@@ -403,7 +407,7 @@ def a3po_train_step(hidden, w, targets, behav_logp, versions, current_version, a
                   (loss, "loss"), (grad_w, "grad_w")):
         _want(t, torch.float32, nm)
     _want(stats, torch.uint8, "stats"); _want(status, torch.int32, "status"); _want(ws, torch.uint8, "ws")
-    _want(entropy, torch.float32, "entropy")
+    _want(entropy, torch.float32, "entropy"); _want(loss_scale, torch.float32, "loss_scale")
     n, h = hidden.shape
     v = w.shape[0]
     if w.shape[1] != h or grad_w.shape != w.shape or grad_hidden.shape != hidden.shape:
@@ -416,8 +420,29 @@ def a3po_train_step(hidden, w, targets, behav_logp, versions, current_version, a
         _ptr(hidden), _ptr(targets), _ptr(behav_logp), _ptr(versions), _ptr(adv), _ptr(mask), n, h, v, dt,
         int(current_version), float(clip_eps), float(inv_temperature), _ptr(w), _ptr(grad_w),
         int(bool(accumulate_grad_w)), _ptr(grad_hidden), _ptr(logp), _ptr(lse), _ptr(entropy), _ptr(grad_logp),
-        _ptr(loss), _ptr(stats), _ptr(ws), ws.numel(), _ptr(status), _stream(stream))
+        _ptr(loss), _ptr(stats), _ptr(loss_scale), _ptr(ws), ws.numel(), _ptr(status), _stream(stream))
     _check("a3po_train_step", rc)
+
+
+# ------------------------------------------------------------------------------ data-parallel helpers
+def a3po_mask_count_workspace_bytes() -> int:
+    return load_library().a3po_mask_count_workspace_bytes()
+
+
+def a3po_mask_count(mask, count, ws, *, stream=None):
+    """count (int64 device tensor, 1 element) = number of non-zero mask bytes."""
+    _want(mask, torch.uint8, "mask"); _want(count, torch.int64, "count"); _want(ws, torch.uint8, "ws")
+    _check("a3po_mask_count", load_library().a3po_mask_count(_ptr(mask), mask.numel(), _ptr(count), _ptr(ws),
+                                                             ws.numel(), _stream(stream)))
+
+
+def a3po_dp_loss_scale(m_local, m_global, scale, *, loss_local=None, weighted_loss=None, stream=None):
+    """scale = M_local / M_global; with loss_local also weighted_loss = scale * loss_local (device scalars)."""
+    _want(m_local, torch.int64, "m_local"); _want(m_global, torch.int64, "m_global")
+    _want(scale, torch.float32, "scale"); _want(loss_local, torch.float32, "loss_local")
+    _want(weighted_loss, torch.float32, "weighted_loss")
+    _check("a3po_dp_loss_scale", load_library().a3po_dp_loss_scale(_ptr(m_local), _ptr(m_global), _ptr(loss_local),
+                                                                   _ptr(scale), _ptr(weighted_loss), _stream(stream)))
 
 
 # ------------------------------------------------------------------------------ whole step, host inputs

@@ -652,8 +652,8 @@ int a3po_train_step(const void* hidden, const int32_t* targets, const float* beh
                     const float* adv, const uint8_t* mask, int64_t N, int H, int V, a3po_dtype dt,
                     int32_t current_version, float clip_eps, float inv_temperature, const void* w, float* grad_w,
                     int accumulate_grad_w, void* grad_hidden, float* logp, float* lse, float* entropy,
-                    float* grad_logp, float* loss, a3po_stats* stats, void* ws, size_t ws_bytes, uint32_t* status,
-                    void* stream_) {
+                    float* grad_logp, float* loss, a3po_stats* stats, const float* loss_scale, void* ws,
+                    size_t ws_bytes, uint32_t* status, void* stream_) {
   A3PO_RETURN_IF(check_lmhead_args(hidden, w, targets, N, H, V, dt, inv_temperature));
   if (!grad_w || !loss || !(clip_eps >= 0.f) ||
       (N > 0 && (!behav_logp || !versions || !adv || !mask || !grad_hidden || !logp || !lse || !grad_logp)))
@@ -667,8 +667,15 @@ int a3po_train_step(const void* hidden, const int32_t* targets, const float* beh
     // three independent calls; the backward recomputes the logits chunk by chunk
     A3PO_RETURN_IF(a3po_token_logprobs_fwd(hidden, w, targets, mask, N, H, V, dt, inv_temperature, logp, lse, entropy,
                                            ws, ws_bytes, status, stream_));
-    A3PO_RETURN_IF(a3po_loss_fwd_bwd(logp, behav_logp, versions, 0, nullptr, 0, current_version, adv, mask, N,
-                                     clip_eps, 1, loss, stats, grad_logp, ws, ws_bytes, stream_));
+    if (loss_scale == nullptr) {
+      A3PO_RETURN_IF(a3po_loss_fwd_bwd(logp, behav_logp, versions, 0, nullptr, 0, current_version, adv, mask, N,
+                                       clip_eps, 1, loss, stats, grad_logp, ws, ws_bytes, stream_));
+    } else {   // a weighted upstream gradient: forward and backward as two calls, the backward takes the weight
+      A3PO_RETURN_IF(a3po_loss_fwd(logp, behav_logp, versions, 0, nullptr, 0, current_version, adv, mask, N, clip_eps,
+                                   loss, stats, ws, ws_bytes, stream_));
+      A3PO_RETURN_IF(a3po_loss_bwd(logp, behav_logp, versions, 0, nullptr, 0, current_version, adv, mask, N, clip_eps,
+                                   1, loss_scale, stats, grad_logp, ws, ws_bytes, stream_));
+    }
     return a3po_token_logprobs_bwd(hidden, w, targets, lse, grad_logp, N, H, V, dt, inv_temperature, grad_hidden,
                                    grad_w, accumulate_grad_w, ws, ws_bytes, status, stream_);
   }
@@ -731,7 +738,7 @@ int a3po_train_step(const void* hidden, const int32_t* targets, const float* beh
     A3PO_RETURN_IF(merge_kept(part_s, part_e, zy, cb.count, c0, rows, splits, inv_temperature, sprime, logp_c, lse_c,
                               entropy ? ent_c : nullptr, status, stream));
     A3PO_RETURN_IF(loss_fwd_bwd_slice(logp_c + c0, behav_c + c0, versions_c + c0, adv_c + c0, mask_c + c0, rows,
-                                      current_version, clip_eps, n_valid, g_c + c0,
+                                      current_version, clip_eps, n_valid, loss_scale, g_c + c0,
                                       partials + static_cast<size_t>(i) * loss_blocks * loss_partial_bytes(),
                                       loss_blocks, stream));
     // the backward's rows: those with a non-zero gradient (clipped tokens drop out), made contiguous in q
@@ -794,7 +801,7 @@ int a3po_train_step_host(const void* h_hidden, const int32_t* h_targets, const f
 
   A3PO_RETURN_IF(a3po_train_step(hidden, targets, behav, versions, adv, mask, N, H, V, dt, current_version, clip_eps,
                                  inv_temperature, d_w, d_grad_w, accumulate_grad_w, d_grad_hidden, logp, lse, nullptr,
-                                 grad_logp, loss, stats, d_ws, ws_bytes, d_status, stream_));
+                                 grad_logp, loss, stats, nullptr, d_ws, ws_bytes, d_status, stream_));
   if (cudaMemcpyAsync(h_loss, loss, sizeof(float), cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
       (h_stats && cudaMemcpyAsync(h_stats, stats, sizeof(a3po_stats), cudaMemcpyDeviceToHost, stream) != cudaSuccess)) {
     cudaGetLastError();

@@ -126,14 +126,16 @@ int finish_batch_outputs(const int* pos, long long n, const float* logp_c, float
                          int h, cudaStream_t stream);
 
 // ---- loss on a slice, for the row-chunked step (loss_kernels.cu) ----
-// Forward + backward of the A-3PO loss on n tokens with M taken from *n_valid; block partials go to
+// Forward + backward of the A-3PO loss on n tokens with M taken from *n_valid and the upstream gradient from
+// *grad_loss (null = 1); block partials go to
 // partials[0 .. blocks) (loss_partial_bytes() each), which loss_finalize_partials sums in index order.
 size_t loss_partial_bytes();
 int loss_max_partials();
 int loss_blocks_for(long long n, int max_blocks);
 int loss_fwd_bwd_slice(const float* logp, const float* behav, const int32_t* versions, const float* adv,
                        const uint8_t* mask, long long n, int32_t current_version, float clip_eps,
-                       const long long* n_valid, float* grad_logp, void* partials, int blocks, cudaStream_t stream);
+                       const long long* n_valid, const float* grad_loss, float* grad_logp, void* partials, int blocks,
+                       cudaStream_t stream);
 int loss_finalize_partials(const void* partials, int count, float* loss, a3po_stats* stats, cudaStream_t stream);
 
 // Launches a one-warp kernel whose bounded wait must expire after timeout_ms and set the status bit.

@@ -330,6 +330,15 @@ __global__ void __launch_bounds__(kLossThreads) mask_count_finalize_kernel(const
   sum_counts_block(block_counts, count, out, sh);
 }
 
+// Data-parallel mean: a shard with M_r valid tokens out of M in the whole job weighs M_r / M.
+__global__ void dp_scale_kernel(const long long* m_local, const long long* m_global, const float* loss_local,
+                                float* scale, float* weighted_loss) {
+  const long long m = *m_global;
+  const float sc = m > 0 ? static_cast<float>(static_cast<double>(*m_local) / static_cast<double>(m)) : 0.f;
+  *scale = sc;
+  if (loss_local) *weighted_loss = sc * *loss_local;
+}
+
 // versions given per sequence: write the per-token array the streaming kernels read.
 __global__ void __launch_bounds__(kLossThreads) expand_versions_kernel(const int32_t* per_seq,
                                                                       const int32_t* cu_seqlens, int b,
@@ -494,13 +503,14 @@ int loss_blocks_for(long long n, int max_blocks) { return grid_for((n + 7) / 8, 
 
 int loss_fwd_bwd_slice(const float* logp, const float* behav, const int32_t* versions, const float* adv,
                        const uint8_t* mask, long long n, int32_t current_version, float clip_eps,
-                       const long long* n_valid, float* grad_logp, void* partials, int blocks, cudaStream_t stream) {
+                       const long long* n_valid, const float* grad_loss, float* grad_logp, void* partials, int blocks,
+                       cudaStream_t stream) {
   LossArgs p;
   p.logp = logp; p.behav = behav; p.versions = versions; p.prox = nullptr; p.adv = adv; p.mask = mask; p.n = n;
   p.current_version = current_version;
   p.lo = 1.0f - clip_eps; p.hi = 1.0f + clip_eps;
   p.detach = 1;
-  p.grad_loss = nullptr;
+  p.grad_loss = grad_loss;
   p.grad_logp = grad_logp;
   p.n_valid_ptr = n_valid;
   const bool vec = aligned_to(logp, 16) && aligned_to(behav, 16) && aligned_to(versions, 16) && aligned_to(adv, 16) &&
@@ -608,6 +618,36 @@ int a3po_loss_fwd_bwd(const float* logp, const float* behav_logp, const int32_t*
   return a3po::run_loss(a3po::kFwdBwd, logp, behav_logp, nullptr, versions, versions_per_seq, cu_seqlens, B,
                         current_version, adv, mask, N, clip_eps, detach_prox, nullptr, nullptr, loss, stats,
                         grad_logp, ws, ws_bytes, stream);
+}
+
+size_t a3po_mask_count_workspace_bytes(void) { return a3po::round_up(sizeof(long long) * a3po::kMaxLossBlocks, 256) + 256; }
+
+int a3po_mask_count(const uint8_t* mask, int64_t N, int64_t* count, void* ws, size_t ws_bytes, void* stream_) {
+  using namespace a3po;
+  if (N < 0 || !count || (N > 0 && !mask)) return A3PO_ERR_INVALID_ARG;
+  if (!ws || !aligned_to(ws, 256) || ws_bytes < a3po_mask_count_workspace_bytes()) return A3PO_ERR_WORKSPACE;
+  if (sm_count() <= 0) return A3PO_ERR_NO_DEVICE;
+  cudaStream_t stream = as_stream(stream_);
+  long long* block_counts = static_cast<long long*>(ws);
+  const int cb = grid_for((N + 15) / 16);
+  A3PO_LAUNCH(kKMaskCount, stream, mask_count_kernel<<<cb, kLossThreads, 0, stream>>>(mask, N, block_counts));
+  A3PO_RETURN_IF(after_launch());
+  A3PO_LAUNCH(kKMaskCountFinalize, stream, mask_count_finalize_kernel<<<1, kLossThreads, 0, stream>>>(
+                                               block_counts, cb, reinterpret_cast<long long*>(count)));
+  return after_launch();
+}
+
+int a3po_dp_loss_scale(const int64_t* m_local, const int64_t* m_global, const float* loss_local, float* scale,
+                       float* weighted_loss, void* stream_) {
+  using namespace a3po;
+  if (!m_local || !m_global || !scale || (loss_local && !weighted_loss)) return A3PO_ERR_INVALID_ARG;
+  if (sm_count() <= 0) return A3PO_ERR_NO_DEVICE;
+  cudaStream_t stream = as_stream(stream_);
+  A3PO_LAUNCH(kKLossFinalize, stream, dp_scale_kernel<<<1, 1, 0, stream>>>(
+                                          reinterpret_cast<const long long*>(m_local),
+                                          reinterpret_cast<const long long*>(m_global), loss_local, scale,
+                                          weighted_loss));
+  return after_launch();
 }
 
 int a3po_decoupled_loss_fwd_bwd(const float* logp, const float* behav_logp, const float* prox_logp, const float* adv,

@@ -175,3 +175,50 @@ def test_keeping_step_in_several_row_chunks():
     _device_step(wl, ref["behav"], part)
     l_many = a3po.a3po_kernel_launch_count() - launches0 - l_one
     assert l_many > l_one                                         # it really ran in more than one chunk
+
+
+@pytest.mark.parametrize("ws_kind", ["recommended", "min"])
+def test_loss_scale_and_data_parallel_helpers(ws_kind):
+    """loss_scale multiplies every gradient and leaves the loss alone (both workspace regimes); the data-parallel
+    wrapper on one rank (M_global = M_local, weight 1) reproduces the plain step; a3po_mask_count and
+    a3po_dp_loss_scale give M and M_r / M."""
+    from paper_2512_06547_b200.data_parallel import gpu_data_parallel_step
+    wl = make("1p5b", dict(V=2048 + 24, H=256, n_prompts=2, group=4, row_len=120, len_lo=30, len_hi=120), False)
+    ref = oracle_step(wl, wl.hidden, wl.w)
+    dt = a3po.A3PO_BF16
+    size = a3po.a3po_train_step_workspace_bytes if ws_kind == "recommended" else a3po.a3po_train_step_min_workspace_bytes
+    ws_bytes = size(wl.N, wl.H, wl.V, dt)
+    plain = _device_step(wl, ref["behav"], ws_bytes)
+    to_dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(DEV)
+    # counts and weights
+    count = torch.zeros(1, dtype=torch.int64, device=DEV)
+    a3po.a3po_mask_count(to_dev(wl.mask), count, a3po.new_workspace(a3po.a3po_mask_count_workspace_bytes()))
+    assert int(count.item()) == int(wl.mask.sum())
+    total = count * 4
+    scale, weighted = torch.zeros(1, device=DEV), torch.zeros(1, device=DEV)
+    a3po.a3po_dp_loss_scale(count, total, scale, loss_local=plain["loss"], weighted_loss=weighted)
+    torch.cuda.synchronize()
+    assert float(scale.item()) == 0.25 and float(weighted.item()) == pytest.approx(0.25 * float(plain["loss"].item()))
+    # the step with that weight
+    n = wl.N
+    out = dict(logp=torch.empty(n, device=DEV), lse=torch.empty(n, device=DEV), grad_logp=torch.empty(n, device=DEV),
+               loss=torch.zeros(1, device=DEV), grad_hidden=torch.empty_like(wl.hidden),
+               grad_w=torch.empty((wl.V, wl.H), dtype=torch.float32, device=DEV))
+    ws = a3po.new_workspace(ws_bytes)
+    a3po.a3po_train_step(wl.hidden, wl.w, to_dev(wl.targets), to_dev(ref["behav"]), to_dev(wl.versions),
+                         wl.current_version, to_dev(wl.adv), to_dev(wl.mask), wl.clip_eps, out["logp"], out["lse"],
+                         out["grad_logp"], out["loss"], out["grad_hidden"], out["grad_w"], ws, loss_scale=scale)
+    torch.cuda.synchronize()
+    assert float(out["loss"].item()) == float(plain["loss"].item())
+    assert torch.allclose(out["grad_logp"], 0.25 * plain["grad_logp"], rtol=1e-6, atol=0)
+    assert rel_fro(to_np64(out["grad_w"]), 0.25 * to_np64(plain["grad_w"])) <= 5e-3        # bf16 roundings differ
+    assert rel_fro(to_np64(out["grad_hidden"]), 0.25 * to_np64(plain["grad_hidden"])) <= 5e-3
+    # the wrapper on a single rank
+    batch = dict(hidden=wl.hidden, w=wl.w, targets=to_dev(wl.targets), behav_logp=to_dev(ref["behav"]),
+                 versions=to_dev(wl.versions), current_version=wl.current_version, adv=to_dev(wl.adv),
+                 mask=to_dev(wl.mask), clip_eps=wl.clip_eps, ws=ws, **out)
+    res = gpu_data_parallel_step()(batch)
+    torch.cuda.synchronize()
+    assert float(res["scale"].item()) == 1.0 and int(res["m_global"].item()) == int(wl.mask.sum())
+    assert float(res["loss"].item()) == pytest.approx(float(plain["loss"].item()), rel=1e-6)
+    assert torch.equal(res["grad_w"], plain["grad_w"]) and torch.equal(res["grad_logp"], plain["grad_logp"])
