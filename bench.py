@@ -633,8 +633,7 @@ def run_loss_sweep(args):
     sampler = ClockSampler(0)
     sampler.start()
     time.sleep(0.3)
-    entry = loss_sweep_entry(args.tokens, sampler, dev, peaks, min_seconds=max(1.5, 0.05 * args.steps),
-                             warmup=args.warmup)
+    entry = loss_sweep_entry(args.tokens, sampler, dev, peaks, min_seconds=args.min_seconds, warmup=args.warmup)
     sampler.stop()
     line = {
         "metric": METRIC, "value": entry["value"], "unit": "tokens/s", "n_gpus": 1, "steps": args.steps,
@@ -665,6 +664,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="8b", choices=sorted(WORKLOAD_TEXT) + ["loss_sweep"])
     ap.add_argument("--tokens", type=int, default=1 << 26, help="token count of --workload loss_sweep")
+    ap.add_argument("--min-seconds", type=float, default=1.5,
+                    help="length of the timed window of --workload loss_sweep (short values for profiler captures)")
     ap.add_argument("--oracle-rows", type=int, default=256)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-configs", action="store_true",

@@ -60,11 +60,14 @@ template <int MT> struct TileCfg {
   static constexpr uint32_t kStageBytes = kAStage + kBBytes;
   static constexpr size_t kSmemBytes = 1024 /*alignment slack*/ + kStages * kStageBytes + 2 * kSlabBytes + 256 /*barriers*/;
 };
-constexpr int kGroupM = 16;
+// Row tiles per rasterisation group (see ItemMap).  Small groups win on B200: with 4 the 8B-shaped step takes
+// 216 ms against 231 with 16 (1.5B-shaped: 10.7 against 11.2 ms), 3 and 6 are worse than 4 and 8; the kernels
+// are energy bound under the board's power cap and fewer HBM re-reads of the operands are fewer joules.
+constexpr int kGroupM = 4;
 
 // Work decomposition: an item is (row tile, vocabulary split); a split is a contiguous range of
 // column tiles.  Items are ordered so that CTAs running at the same time share row tiles and
-// column tiles through L2: groups of kGroupM row tiles, all splits of a group before the next.
+// column tiles through L2: groups of group_m row tiles, all splits of a group before the next.
 struct ItemMap {
   int m_tiles;
   int n_tiles;
@@ -1022,7 +1025,7 @@ int launch_gemm(const Operand& a, const Operand& b, int splits, const typename E
   im.n_tiles = static_cast<int>((b.mn_extent + BN - 1) / BN);
   im.splits = splits > 0 ? splits : im.n_tiles;
   im.items = static_cast<long long>(im.m_tiles) * im.splits;
-  im.group_m = tuning_override("A3PO_GROUP_M", kGroupM);
+  im.group_m = splits > 0 ? tuning_override("A3PO_GROUP_M", kGroupM) : tuning_override("A3PO_GROUP_M_GRAD", kGroupM);
   im.dyn_rows = dyn.rows;
   im.dyn_is_k = dyn.is_k;
   im.zero_when_empty = dyn.zero_when_empty;
@@ -1102,7 +1105,7 @@ int launch_pair_gemm(const Operand& a, const Operand& b, int splits, const typen
   im.n_tiles = static_cast<int>((b.mn_extent + BN - 1) / BN);
   im.splits = splits > 0 ? splits : im.n_tiles;
   im.items = static_cast<long long>(im.m_tiles) * im.splits;
-  im.group_m = tuning_override("A3PO_GROUP_M", kGroupM / 2);
+  im.group_m = tuning_override("A3PO_GROUP_M", kGroupM);
   im.dyn_rows = dyn.rows;
   im.dyn_is_k = 0;
   im.zero_when_empty = 0;
