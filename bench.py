@@ -40,15 +40,17 @@ if ROOT not in sys.path:
 
 METRIC = "logprob+A-3PO loss fwd/bwd tokens/s; % of bf16 TC peak & HBM roofline"
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant GEMM kernel, from the ncu captures
-# summarised under profiles/: bytes per row that takes part, taken on a --small case of the same H and V and
-# scaled by the rows of the launch (W re-reads and the kept matrix both grow with the rows).  An entry is
-# None until a capture of the current kernel exists for that shape.
-NCU_TRAFFIC_PER_ROW = {
-    # (H, V): {kernel name: bytes per row}
+# dram__bytes_read.sum + dram__bytes_write.sum of the dominant GEMM kernel (the forward that keeps the softmax), from
+# the one-pass ncu captures of the full-size launches summarised in profiles/step_8b_launch_list_and_dram.md: bytes
+# per step over all its launches of the step (the row chunks); divided by the launches of a step for the per-launch
+# figure.  Reset an entry to None when the kernel or its rasterisation changes.
+NCU_TRAFFIC_PER_STEP = {
+    "8b": {"gemm_tn<fwd_logsoftmax+keep>": 56.03e9 + 19.90e9 + 13.62e9 + 4.43e9},
+    "1p5b": {"gemm_tn<fwd_logsoftmax+keep>": 3.62e9 + 2.75e9},
 }
-# Loss kernels (profiles/loss_kernels_16Mi_tokens_ncu_full.md): bytes per token at N = 2^24.
-NCU_TRAFFIC_PER_TOKEN_LOSS = {"loss_fwd_bwd": (285.231616e6 + 40.569600e6) / 16777216}
+# Fused loss kernel (profiles/loss_kernel_16Mi_tokens_ncu_full.md): DRAM bytes per token at N = 2^24 (17 B read exactly;
+# most of the 4 B of gradient written per token is still in L2 when the kernel ends).
+NCU_TRAFFIC_PER_TOKEN_LOSS = {"loss_fwd_bwd": (285.257e6 + 21.87e6) / 16777216}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 LONG_REGION_S = 2.0      # a timed region longer than this runs under the power cap: the sustained peak applies
 
@@ -226,7 +228,7 @@ def reduce_over_ranks(times_ms, counts, device):
     return t.tolist(), c.tolist()
 
 
-def tensor_roofline(kernels, steps, h, v, region_s, peaks):
+def tensor_roofline(kernels, steps, h, v, region_s, peaks, workload=None, small=False):
     """Roofline object of the dominant GEMM kernel.  The peak is the measured cuBLAS bf16 figure that matches the
     timed region: the burst figure for a short region, the sustained one when the region is long enough for the
     board to sit at its power cap."""
@@ -239,14 +241,17 @@ def tensor_roofline(kernels, steps, h, v, region_s, peaks):
     burst = peaks["bf16_tflops"]
     long_region = region_s > LONG_REGION_S
     peak = sustained if long_region else burst
-    per_row = NCU_TRAFFIC_PER_ROW.get((h, v), {}).get(dom["kernel"])
+    per_step = None if small else NCU_TRAFFIC_PER_STEP.get(workload, {}).get(dom["kernel"])
     launches_per_step = max(dom["launches"] // max(steps, 1), 1)
     all_flops = sum(2.0 * k["rows"] * v * h * steps for k in gemms)
     all_ms = sum(k["ms_total"] for k in gemms)
     return {"bound": "tensor", "kernel": dom["kernel"], "achieved": dom["tflops"], "peak": peak,
             "unit": "TFLOP/s", "frac": round(dom["tflops"] / peak, 4),
-            "traffic": round(per_row * dom["rows"] / launches_per_step) if per_row else None,
+            "traffic": round(per_step / launches_per_step) if per_step else None,
             "algorithmic_flops_per_launch": 2.0 * dom["rows"] * v * h / launches_per_step,
+            # the keeping forward: hidden rows in, 2 bytes per (row, vocabulary entry) out, W once
+            "algorithmic_bytes_per_launch": (round((dom["rows"] * (2.0 * h + 2.0 * ((v + 7) // 8 * 8)) + 2.0 * v * h)
+                                                   / launches_per_step) if "keep" in dom["kernel"] else None),
             "launches_per_step": launches_per_step,
             "peak_source": "%s cuBLAS bf16, %s (timed region %.1f s)" % (
                 peaks["_source"], "sustained" if long_region else "burst", region_s),
@@ -418,7 +423,7 @@ def secondary_step_config(name, args, sampler, dev, barrier, peaks):
                            with_e2e=False)
     kernels, step_flops = kernel_table(r["per_kernel"], steps, r["n_valid"], r["bwd_rows"], r["n"], r["v"], r["h"])
     ms_per_step = r["ms_total"] / steps
-    roof = tensor_roofline(kernels, steps, r["h"], r["v"], r["ms_total"] * 1e-3, peaks)
+    roof = tensor_roofline(kernels, steps, r["h"], r["v"], r["ms_total"] * 1e-3, peaks, workload=name)
     torch.cuda.empty_cache()
     return {"workload": WORKLOAD_TEXT[name], "rows": r["n"], "valid_tokens": r["n_valid"], "steps": steps,
             "ms_per_step": round(ms_per_step, 4), "value": round(r["n_valid"] / (ms_per_step * 1e-3), 1),
@@ -426,7 +431,8 @@ def secondary_step_config(name, args, sampler, dev, barrier, peaks):
             "workspace_gib": round(r["ws_bytes"] / 2 ** 30, 2),
             "recompute_free": not any(k["kernel"] == "gemm_tn<dz>" for k in kernels),
             "roofline": {k: roof[k] for k in ("bound", "kernel", "achieved", "peak", "unit", "frac", "frac_of_burst",
-                                              "frac_of_sustained", "peak_source") if k in roof},
+                                              "frac_of_sustained", "peak_source", "traffic",
+                                              "algorithmic_bytes_per_launch") if k in roof},
             "kernels": [{k: e[k] for k in ("kernel", "ms_total", "share", "tflops") if k in e} for e in kernels[:4]],
             "clocks": r["clocks"]}
 
@@ -469,7 +475,8 @@ def run_ours(args):
     value = total_valid * args.steps / (ms_total * 1e-3)
     e2e_value = total_valid * args.steps / (e2e_ms_total * 1e-3)
     kernels, step_flops = kernel_table(r["per_kernel"], args.steps, n_valid, r["bwd_rows"], n, v, h)
-    roofline = tensor_roofline(kernels, args.steps, h, v, ms_total * 1e-3, peaks)
+    roofline = tensor_roofline(kernels, args.steps, h, v, ms_total * 1e-3, peaks, workload=args.workload,
+                               small=args.small or args.separate_calls)
 
     # ---- the other named configurations, each in its own window (one GPU only)
     configs = None
