@@ -84,7 +84,10 @@ int a3po_version(void);
  * logp, lse: fp32 [N] outputs (lse is needed by the backward).
  * entropy: fp32 [N] or NULL; when given, receives the policy entropy -sum_v p_v log p_v of
  *          each row (the diagnostic of Fig. 4), computed in the same vocabulary sweep.
- * ws/ws_bytes: at least a3po_token_logprobs_workspace_bytes(N,H,V,dt,0).
+ * ws/ws_bytes: at least a3po_token_logprobs_min_workspace_bytes(N,H,V,dt,0).  With the larger
+ * a3po_token_logprobs_workspace_bytes(N,H,V,dt,0) (bf16 inputs, row_mask given) the rows with
+ * row_mask != 0 are gathered first and only they are multiplied; with less than that every row is
+ * computed and the masked ones are discarded afterwards (same results, more work).
  * ------------------------------------------------------------------------------------------ */
 size_t a3po_token_logprobs_workspace_bytes(int64_t N, int H, int V, a3po_dtype dt, int is_bwd);
 
@@ -106,7 +109,9 @@ int a3po_token_logprobs_fwd(const void* hidden, const void* w, const int32_t* ta
  * training step, Sec. 4.1); 0 overwrites it.
  * dz is materialised only for a chunk of rows at a time inside `ws` (bf16 for A3PO_BF16);
  * the chunk length adapts to ws_bytes.  a3po_token_logprobs_workspace_bytes(...,1) returns
- * the size that lets the library use its preferred chunk; the call fails with
+ * the size that lets the library use its preferred chunk AND gather the rows with a non-zero
+ * grad_logp first (bf16 inputs), so that padding and clipped tokens cost nothing; with less
+ * than that they are multiplied as zero rows (same results, more work).  The call fails with
  * A3PO_ERR_WORKSPACE below a3po_token_logprobs_min_workspace_bytes(...).
  * ------------------------------------------------------------------------------------------ */
 size_t a3po_token_logprobs_min_workspace_bytes(int64_t N, int H, int V, a3po_dtype dt, int is_bwd);

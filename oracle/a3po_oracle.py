@@ -37,6 +37,7 @@ __all__ = [
     "loss_terms",
     "loss_fwd",
     "loss_bwd",
+    "decoupled_loss",
     "grpo_advantages",
 ]
 
