@@ -85,6 +85,10 @@ struct ItemMap {
   // does its work only if *select == select_value (the other one then exits at once).
   const int* select;
   int select_value;
+  // Optional pacing of the CTAs of a launch (see Pace): ring of arrival counters, null = off.
+  unsigned int* pace;
+  int pace_period;  // k-blocks between two pacing points
+  int pace_slack;   // how many pacing points a CTA may be ahead of the slowest one
 };
 
 struct Item {
@@ -114,6 +118,65 @@ __device__ __forceinline__ Item decode_item(const ItemMap& im, long long i) {
   it.n_end = static_cast<int>(static_cast<long long>(it.split + 1) * im.n_tiles / im.splits);
   return it;
 }
+
+// Pacing.  The CTAs of a launch that run at the same time read the same operand tiles (that is what the item order
+// arranges), but only the first reader of a tile takes it from HBM if the others follow before L2 has replaced
+// it.  Nothing keeps a persistent CTA in step with the others over dozens of tiles, so they drift apart and the
+// same bytes come out of HBM several times: on the 8B-shaped batch the gradient contractions read 100 GB per
+// launch unpaced and 51 GB paced (the floor for 148 concurrent 256 x 256 tiles), 5-8 % of their time under the
+// board's power cap.  Every kPacePeriod k-blocks the producer thread of each CTA counts itself in at a pacing
+// point and does not run more than kPaceSlack points ahead of the slowest CTA.  It is advisory: no data depends
+// on it, a wait gives up after kPaceWaitCycles and the CTA then skips a growing number of points (so CTAs that
+// cannot be in step, e.g. because they started late, lose microseconds, not the kernel), and a CTA with nothing
+// to load counts itself in for the points it will not reach.
+// Counters of one launch: kPaceRing arrival counters (point g uses slot g mod kPaceRing; a slot counts up over the
+// launch) followed by one counter of finished CTAs; the last CTA to finish zeroes all of them again, so a block of
+// counters is zero whenever no launch is using it.
+constexpr int kPaceRing = 32;
+constexpr int kPaceBlockWords = 64;            // one launch's counters: ring + finished count, padded to 256 bytes
+constexpr int kPaceBlocks = 32;                // handed out round-robin, so launches on different streams differ
+constexpr int kPacePeriod = 8;
+constexpr int kPaceSlack = 2;
+constexpr long long kPaceWaitCycles = 40000;   // 20-40 us
+struct Pace {
+  unsigned int* slots = nullptr;
+  unsigned int ctas = 0;
+  int slack = 0;
+  int skip = 0;
+  int backoff = 8;
+  long long next = 0;   // index of the next pacing point of this CTA
+
+  __device__ __forceinline__ void arrive() {
+    atomicAdd(&slots[next & (kPaceRing - 1)], 1u);
+    ++next;
+  }
+  __device__ __forceinline__ void arrive_and_wait() {
+    const long long behind = next - slack;
+    arrive();
+    if (behind < 0) return;
+    if (skip > 0) { --skip; return; }
+    const unsigned int expected = static_cast<unsigned int>(behind / kPaceRing + 1) * ctas;
+    volatile unsigned int* slot = slots + (behind & (kPaceRing - 1));
+    if (*slot < expected) {
+      const long long t0 = clock64();
+      while (*slot < expected) {
+        if (clock64() - t0 > kPaceWaitCycles) {
+          skip = backoff;
+          backoff = backoff < 4096 ? 2 * backoff : backoff;
+          return;
+        }
+      }
+    }
+    backoff = 8;
+  }
+  __device__ __forceinline__ void finish() {
+    __threadfence();
+    const unsigned int done = atomicAdd(&slots[kPaceRing], 1u);
+    if (done + 1 == ctas) {
+      for (int i = 0; i <= kPaceRing; ++i) slots[i] = 0u;
+    }
+  }
+};
 
 __device__ __forceinline__ float bits_to_float(uint32_t u) { return __uint_as_float(u); }
 
@@ -622,10 +685,24 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     if (elect_one()) {
       int stage = 0;
       uint32_t phase = 0;
+      // pacing points: every CTA of the launch passes the same number per wave of items, whether it has an item
+      // in that wave (or a last column tile in its item) or not
+      Pace pace;
+      const bool paced = im.pace != nullptr && im.pace_period > 0 && im.items > 0 && k_blocks > 0;
+      const int points_per_tile = paced ? (k_blocks + im.pace_period - 1) / im.pace_period : 0;
+      const long long points_per_wave =
+          static_cast<long long>((im.n_tiles + im.splits - 1) / im.splits) * points_per_tile;
+      long long waves_done = 0;
+      if (paced) {
+        pace.slots = im.pace;
+        pace.ctas = gridDim.x;
+        pace.slack = im.pace_slack;
+      }
       for (long long i = blockIdx.x; i < im.items && ok; i += gridDim.x) {
         const Item it = decode_item(im, i);
         for (int nt = it.n_begin; nt < it.n_end && ok; ++nt) {
           for (int kb = 0; kb < k_blocks; ++kb) {
+            if (paced && kb % im.pace_period == 0) pace.arrive_and_wait();
             if (!A3PO_TIMED_WAIT(waited, mbar_wait(&empty_bar[stage], phase ^ 1u, abort_flag))) { ok = false; break; }
             mbar_arrive_expect_tx(&full_bar[stage], kStageBytes);
             uint8_t* sa = smem_a + stage * kAStage;
@@ -647,6 +724,14 @@ gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             if (++stage == kStages) { stage = 0; phase ^= 1u; }
           }
         }
+        ++waves_done;
+        if (paced)
+          while (pace.next < waves_done * points_per_wave) pace.arrive();
+      }
+      if (paced) {
+        const long long waves = (im.items + gridDim.x - 1) / gridDim.x;
+        while (pace.next < waves * points_per_wave) pace.arrive();
+        pace.finish();
       }
     }
   } else if (warp == 1) {
@@ -1000,6 +1085,31 @@ int tuning_override(const char* name, int fallback) {
 #endif
 }
 
+// Pacing counters (see Pace) live in the library's device image, 8 KB per GPU: all zero when the library is
+// loaded, and every paced launch leaves its block zero again.  In host code the array's name is only a handle for
+// cudaGetSymbolAddress.
+__device__ __align__(256) unsigned int g_pace_counters[kPaceBlocks * kPaceBlockWords];
+unsigned int* next_pace_block() {
+  static std::mutex mu;
+  static unsigned int* cached[64];
+  static unsigned int turn[64];
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
+    cudaGetLastError();
+    return nullptr;
+  }
+  std::lock_guard<std::mutex> lock(mu);
+  if (!cached[dev]) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_pace_counters) != cudaSuccess || !p) {
+      cudaGetLastError();
+      return nullptr;   // the launch then runs unpaced
+    }
+    cached[dev] = static_cast<unsigned int*>(p);
+  }
+  return cached[dev] + static_cast<size_t>(turn[dev]++ % kPaceBlocks) * kPaceBlockWords;
+}
+
 // Device-resident row count for a launch (see ItemMap).
 struct DynRows {
   const int* rows = nullptr;
@@ -1033,6 +1143,10 @@ int launch_gemm(const Operand& a, const Operand& b, int splits, const typename E
   im.dyn_cap = dyn.cap;
   im.select = dyn.select;
   im.select_value = dyn.select_value;
+  im.pace_period = tuning_override("A3PO_PACE_PERIOD", kPacePeriod);
+  im.pace_slack = tuning_override("A3PO_PACE_SLACK", kPaceSlack);
+  if (im.pace_slack > kPaceRing / 2) im.pace_slack = kPaceRing / 2;   // a slot must not be reused while waited on
+  im.pace = tuning_override("A3PO_PACE_OFF", 0) == 1 ? nullptr : next_pace_block();
   const int k_blocks = static_cast<int>((a.k_extent + BK - 1) / BK);
   auto kernel = gemm_tn_kernel<Epi, A_MN, B_MN, MT>;
   if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemBytes)) !=
@@ -1113,6 +1227,9 @@ int launch_pair_gemm(const Operand& a, const Operand& b, int splits, const typen
   im.dyn_cap = dyn.cap;
   im.select = nullptr;
   im.select_value = 0;
+  im.pace = nullptr;
+  im.pace_period = 0;
+  im.pace_slack = 0;
   const int k_blocks = static_cast<int>((a.k_extent + BK - 1) / BK);
   long long pairs = pairs_max;
   if (pairs > im.items) pairs = im.items;

@@ -1,5 +1,6 @@
 """The kernel variants that only a tuning build (-DA3PO_TUNING) can select stay correct: the forward on CTA pairs
-(tcgen05 cta_group::2) and the gradient contractions on 128 x 256 tiles.  Each variant runs in a child process,
+(tcgen05 cta_group::2), the gradient contractions on 128 x 256 tiles, and the persistent CTAs unpaced or paced at
+every k-block.  Each variant runs in a child process,
 because the switches are environment variables read by the tuning library."""
 import os
 import subprocess
@@ -57,7 +58,8 @@ CHILD = textwrap.dedent("""
 """)
 
 
-@pytest.mark.parametrize("env", [{"A3PO_FWD_PAIR": "1"}, {"A3PO_GRAD_MT": "1"}, {"A3PO_GRAD_MT": "2", "A3PO_FWD_PAIR": "1"}])
+@pytest.mark.parametrize("env", [{"A3PO_FWD_PAIR": "1"}, {"A3PO_GRAD_MT": "1"}, {"A3PO_GRAD_MT": "2", "A3PO_FWD_PAIR": "1"},
+                                 {"A3PO_PACE_OFF": "1"}, {"A3PO_PACE_PERIOD": "1", "A3PO_PACE_SLACK": "1"}])
 def test_tuning_variants_match_the_oracle(env):
     lib = a3po_build.build(tuning=True)
     child_env = dict(os.environ, **env)
