@@ -45,8 +45,8 @@ METRIC = "logprob+A-3PO loss fwd/bwd tokens/s; % of bf16 TC peak & HBM roofline"
 # per step over all its launches of the step (the row chunks); divided by the launches of a step for the per-launch
 # figure.  Reset an entry to None when the kernel or its rasterisation changes.
 NCU_TRAFFIC_PER_STEP = {
-    "8b": {"gemm_tn<fwd_logsoftmax+keep>": 56.03e9 + 19.90e9 + 13.62e9 + 4.43e9},
-    "1p5b": {"gemm_tn<fwd_logsoftmax+keep>": 3.62e9 + 2.75e9},
+    "8b": {"gemm_tn<fwd_logsoftmax+keep>": 21.48e9 + 19.90e9 + 5.90e9 + 4.43e9},
+    "1p5b": {"gemm_tn<fwd_logsoftmax+keep>": 0.70e9 + 2.72e9},
 }
 # Fused loss kernel (profiles/loss_kernel_16Mi_tokens_ncu_full.md): DRAM bytes per token at N = 2^24 (17 B read exactly;
 # most of the 4 B of gradient written per token is still in L2 when the kernel ends).
@@ -249,9 +249,10 @@ def tensor_roofline(kernels, steps, h, v, region_s, peaks, workload=None, small=
             "unit": "TFLOP/s", "frac": round(dom["tflops"] / peak, 4),
             "traffic": round(per_step / launches_per_step) if per_step else None,
             "algorithmic_flops_per_launch": 2.0 * dom["rows"] * v * h / launches_per_step,
-            # the keeping forward: hidden rows in, 2 bytes per (row, vocabulary entry) out, W once
-            "algorithmic_bytes_per_launch": (round((dom["rows"] * (2.0 * h + 2.0 * ((v + 7) // 8 * 8)) + 2.0 * v * h)
-                                                   / launches_per_step) if "keep" in dom["kernel"] else None),
+            # the keeping forward: hidden rows in, 2 bytes per (row, vocabulary entry) out, W once per launch
+            "algorithmic_bytes_per_launch": (round(dom["rows"] * (2.0 * h + 2.0 * ((v + 7) // 8 * 8))
+                                                   / launches_per_step + 2.0 * v * h)
+                                             if "keep" in dom["kernel"] else None),
             "launches_per_step": launches_per_step,
             "peak_source": "%s cuBLAS bf16, %s (timed region %.1f s)" % (
                 peaks["_source"], "sustained" if long_region else "burst", region_s),

@@ -262,7 +262,7 @@ size_t a3po_token_logprobs_min_workspace_bytes(int64_t N, int H, int V, a3po_dty
   if (!is_bwd) {
     size_t a = fwd_ws_for(N, simt_fwd_splits(N, V));
     if (dt == A3PO_BF16) {
-      const size_t b = fwd_ws_for(N, lmhead_tc_fwd_splits(N, V));
+      const size_t b = fwd_ws_for(N, lmhead_tc_fwd_splits(N, H, V));
       if (b > a) a = b;
     }
     return a;
@@ -297,7 +297,7 @@ int a3po_token_logprobs_fwd(const void* hidden, const void* w, const int32_t* ta
   if (!ws || !aligned_to(ws, 256)) return A3PO_ERR_WORKSPACE;
   cudaStream_t stream = as_stream(stream_);
   const bool tc = use_tc(dt, hidden, w, N, H, V);
-  const int splits = tc ? lmhead_tc_fwd_splits(N, V) : simt_fwd_splits(N, V);
+  const int splits = tc ? lmhead_tc_fwd_splits(N, H, V) : simt_fwd_splits(N, V);
   if (ws_bytes < fwd_ws_for(N, splits)) return A3PO_ERR_WORKSPACE;
   // Masked rows are skipped, not computed: with a row mask and enough workspace the kept rows are
   // gathered into a compact buffer and the kernels run on that (count stays on the device).
@@ -435,7 +435,7 @@ constexpr size_t kScanBytes = 2 * 4096 * sizeof(int);  // block counts + offsets
 
 size_t fwd_keep_ws_bytes(long long n, int h, int v) {
   const size_t cap = static_cast<size_t>(compact_capacity(n));
-  const int splits = lmhead_tc_fwd_splits(static_cast<long long>(cap), v);
+  const int splits = lmhead_tc_fwd_splits(static_cast<long long>(cap), h, v);
   return round_up(kScanBytes, 256) + round_up(cap * static_cast<size_t>(h) * 2, 256) /*hidden_c*/ +
          4 * round_up(sizeof(float) * cap, 256) /*zy, logp_c, lse_c, ent_c*/ +
          2 * round_up(sizeof(float) * cap * splits, 256) /*part_s, part_e*/ + 256;
@@ -477,7 +477,7 @@ int a3po_token_logprobs_fwd_keep(const void* hidden, const void* w, const int32_
   const KeptLayout kl = kept_layout(N, V);
   char* kb = static_cast<char*>(kept);
   const long long cap = compact_capacity(N);
-  const int splits = lmhead_tc_fwd_splits(cap, V);
+  const int splits = lmhead_tc_fwd_splits(cap, H, V);
 
   Arena arena(ws, ws_bytes);
   CompactBuffers cb;
@@ -730,7 +730,7 @@ int a3po_train_step(const void* hidden, const int32_t* targets, const float* beh
   for (int i = 0; i < n_chunks; ++i) {
     const long long c0 = static_cast<long long>(i) * chunk_rows;
     const long long rows = (c0 + chunk_rows <= cap) ? chunk_rows : cap - c0;
-    const int splits = lmhead_tc_fwd_splits(rows, V);
+    const int splits = lmhead_tc_fwd_splits(rows, H, V);
     A3PO_RETURN_IF(gather_rows_range(hidden, H, cb.idx, cb.count, c0, rows, cb.hidden_c, stream));
     A3PO_RETURN_IF(target_logits(hidden_c, w, cb.targets_c, cb.count, c0, rows, H, V, inv_temperature, zy, stream));
     A3PO_RETURN_IF(lmhead_fwd_keep_tc(hidden_c, w, cb.targets_c + c0, zy + c0, rows, H, V, inv_temperature,

@@ -53,7 +53,7 @@ int scatter_rows(const void* src_c, int h, const int* pos, long long n, void* ds
 // ---- tcgen05 / TMEM / TMA kernels (lmhead_tc.cu), bf16 only ----
 bool lmhead_tc_supported(const void* hidden, const void* w, long long n, int h, int v);
 // Vocabulary splits the tensor-core forward wants for (n, v): each (row tile, split) pair is one work item.
-int lmhead_tc_fwd_splits(long long n, int v);
+int lmhead_tc_fwd_splits(long long n, int h, int v);
 // `dyn_rows` (device, may be null): number of rows of `hidden` that are really present (compact row space);
 // partials are laid out [split][n] regardless.
 int lmhead_fwd_tc(const void* hidden, const void* w, const int32_t* targets, long long n, int h, int v, float inv_t,

@@ -60,10 +60,13 @@ template <int MT> struct TileCfg {
   static constexpr uint32_t kStageBytes = kAStage + kBBytes;
   static constexpr size_t kSmemBytes = 1024 /*alignment slack*/ + kStages * kStageBytes + 2 * kSlabBytes + 256 /*barriers*/;
 };
-// Row tiles per rasterisation group (see ItemMap).  Small groups win on B200: with 4 the 8B-shaped step takes
-// 216 ms against 231 with 16 (1.5B-shaped: 10.7 against 11.2 ms), 3 and 6 are worse than 4 and 8; the kernels
-// are energy bound under the board's power cap and fewer HBM re-reads of the operands are fewer joules.
+// Row tiles per rasterisation group (see ItemMap) of the contractions whose items are single output tiles (the
+// gradients).  Small groups win on B200: with 4 the 8B-shaped step takes 216 ms against 231 with 16 (1.5B-shaped:
+// 10.7 against 11.2 ms), 3 and 6 are worse than 4 and 8; the kernels are energy bound under the board's power cap
+// and fewer HBM re-reads of the operands are fewer joules.
 constexpr int kGroupM = 4;
+// The forward contractions (items sweep a range of column tiles) take large groups instead, see fwd_group_m().
+constexpr long long kFwdGroupBytes = 40ll << 20;
 
 // Work decomposition: an item is (row tile, vocabulary split); a split is a contiguous range of
 // column tiles.  Items are ordered so that CTAs running at the same time share row tiles and
@@ -135,8 +138,8 @@ __device__ __forceinline__ Item decode_item(const ItemMap& im, long long i) {
 constexpr int kPaceRing = 32;
 constexpr int kPaceBlockWords = 64;            // one launch's counters: ring + finished count, padded to 256 bytes
 constexpr int kPaceBlocks = 32;                // handed out round-robin, so launches on different streams differ
-constexpr int kPacePeriod = 8;
-constexpr int kPaceSlack = 2;
+constexpr int kPacePeriod = 16;
+constexpr int kPaceSlack = 3;
 constexpr long long kPaceWaitCycles = 40000;   // 20-40 us
 struct Pace {
   unsigned int* slots = nullptr;
@@ -144,30 +147,43 @@ struct Pace {
   int slack = 0;
   int skip = 0;
   int backoff = 8;
-  long long next = 0;   // index of the next pacing point of this CTA
+  unsigned int seen = 0;   // arrivals counted, one point ago, at the point this CTA has to wait for next
+  long long next = 0;      // index of the next pacing point of this CTA
 
   __device__ __forceinline__ void arrive() {
     atomicAdd(&slots[next & (kPaceRing - 1)], 1u);
     ++next;
   }
+  // The counter this CTA will compare at its next pacing point is read one point early (`seen`), so that the
+  // producer does not sit out an L2 round trip at every point; a stale value can only be too small, and then the
+  // loop below reads the counter afresh.
   __device__ __forceinline__ void arrive_and_wait() {
     const long long behind = next - slack;
     arrive();
-    if (behind < 0) return;
-    if (skip > 0) { --skip; return; }
-    const unsigned int expected = static_cast<unsigned int>(behind / kPaceRing + 1) * ctas;
-    volatile unsigned int* slot = slots + (behind & (kPaceRing - 1));
-    if (*slot < expected) {
-      const long long t0 = clock64();
-      while (*slot < expected) {
-        if (clock64() - t0 > kPaceWaitCycles) {
-          skip = backoff;
-          backoff = backoff < 4096 ? 2 * backoff : backoff;
-          return;
+    if (behind >= 0) {
+      if (skip > 0) {
+        --skip;
+      } else {
+        const unsigned int expected = static_cast<unsigned int>(behind / kPaceRing + 1) * ctas;
+        if (seen < expected) {
+          volatile unsigned int* slot = slots + (behind & (kPaceRing - 1));
+          const long long t0 = clock64();
+          bool late = false;
+          while (*slot < expected) {
+            if (clock64() - t0 > kPaceWaitCycles) { late = true; break; }
+          }
+          if (late) {
+            skip = backoff;
+            backoff = backoff < 4096 ? 2 * backoff : backoff;
+          } else {
+            backoff = 8;
+          }
+        } else {
+          backoff = 8;
         }
       }
     }
-    backoff = 8;
+    if (behind + 1 >= 0) seen = *(static_cast<volatile unsigned int*>(slots) + ((behind + 1) & (kPaceRing - 1)));
   }
   __device__ __forceinline__ void finish() {
     __threadfence();
@@ -1110,6 +1126,20 @@ unsigned int* next_pace_block() {
   return cached[dev] + static_cast<size_t>(turn[dev]++ % kPaceBlocks) * kPaceBlockWords;
 }
 
+// Row tiles per group for the forward contractions.  With G row tiles per group the CTAs of a launch work on
+// SMs / G vocabulary splits of the same G row tiles at a time (items are split-major inside a group): every W tile
+// comes out of HBM once per G row tiles, and the G row tiles of the other operand (G x 128 x K x 2 bytes) have to
+// stay in L2 while the column tiles are swept.  G = the largest of SMs, SMs/2, SMs/4, ... whose row tiles fit
+// kFwdGroupBytes.  Measured on the 8B-shaped batch (K = 4096, 65,536 rows, paced CTAs), HBM bytes read by one
+// launch: G = 4: 58 GB, 16: 50 GB, 37: 23 GB, 74: 155 GB (the row tiles no longer fit).
+int fwd_group_m(long long k_extent) {
+  const long long tile_bytes = static_cast<long long>(BM) * k_extent * 2;
+  int g = sm_count();
+  if (g <= 0) g = 148;
+  while (g > kGroupM && g * tile_bytes > kFwdGroupBytes) g /= 2;
+  return g > kGroupM ? g : kGroupM;
+}
+
 // Device-resident row count for a launch (see ItemMap).
 struct DynRows {
   const int* rows = nullptr;
@@ -1135,7 +1165,8 @@ int launch_gemm(const Operand& a, const Operand& b, int splits, const typename E
   im.n_tiles = static_cast<int>((b.mn_extent + BN - 1) / BN);
   im.splits = splits > 0 ? splits : im.n_tiles;
   im.items = static_cast<long long>(im.m_tiles) * im.splits;
-  im.group_m = splits > 0 ? tuning_override("A3PO_GROUP_M", kGroupM) : tuning_override("A3PO_GROUP_M_GRAD", kGroupM);
+  im.group_m = splits > 0 ? tuning_override("A3PO_GROUP_M", fwd_group_m(a.k_extent))
+                          : tuning_override("A3PO_GROUP_M_GRAD", kGroupM);
   im.dyn_rows = dyn.rows;
   im.dyn_is_k = dyn.is_k;
   im.zero_when_empty = dyn.zero_when_empty;
@@ -1342,8 +1373,10 @@ bool fwd_uses_pairs() {
 
 // Picks the number of vocabulary splits so that (row tiles x splits) items spread evenly over
 // the workers (SMs, or CTA pairs with 256-row tiles; static round-robin) while every item still sweeps several
-// column tiles.
-int lmhead_tc_fwd_splits(long long n, int v) {
+// column tiles.  With G row tiles per group and SMs / G splits in flight, a split count that is a multiple of
+// SMs / G makes every full group a whole number of waves, so that the CTAs never hold the row tiles of two
+// groups at once (8B-shaped batch, 65,536 rows: 23 GB read from HBM per launch against 47 GB with 13 splits).
+int lmhead_tc_fwd_splits(long long n, int h, int v) {
   const bool pairs = fwd_uses_pairs();
   const int tile_rows = pairs ? 2 * BM : BM;
   const long long m_tiles = (n + tile_rows - 1) / tile_rows;
@@ -1355,16 +1388,21 @@ int lmhead_tc_fwd_splits(long long n, int v) {
   if (forced > 0) return forced < n_tiles ? (forced < 64 ? forced : 64) : n_tiles;
   const int s_max = n_tiles < 64 ? n_tiles : 64;
   int s_min = s_max < 8 ? s_max : 8;  // several splits in flight keep the row-tile working set inside L2
-  int best = s_min;
+  int step = 1;
+  if (!pairs) {
+    const int group = tuning_override("A3PO_GROUP_M", fwd_group_m(h));
+    if (group > kGroupM && m_tiles >= group && workers % group == 0 && workers / group <= s_max) step = workers / group;
+  }
+  int best = 0;
   double best_cost = 1e300;
-  for (int s = s_min; s <= s_max; ++s) {
+  for (int s = (s_min + step - 1) / step * step; s <= s_max; s += step) {
     const long long items = m_tiles * s;
     const long long waves = (items + workers - 1) / workers;
     const long long tiles_per_item = (n_tiles + s - 1) / s;
     const double cost = static_cast<double>(waves) * (static_cast<double>(tiles_per_item) + 0.5);
     if (cost < best_cost - 1e-9) { best_cost = cost; best = s; }
   }
-  return best;
+  return best > 0 ? best : s_min;
 }
 
 int lmhead_fwd_tc(const void* hidden, const void* w, const int32_t* targets, long long n, int h, int v, float inv_t,
