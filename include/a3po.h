@@ -10,6 +10,9 @@
  *   - Pointers are DEVICE pointers owned by the caller.  The library allocates no device
  *     memory: scratch space is the caller's `ws` buffer (size it with the *_workspace_bytes
  *     functions; 256-byte aligned).  Contents of `ws` are undefined before and after a call.
+ *     Besides that, the library's device image holds two fixed arrays per GPU: 8 KB of
+ *     counters with which the CTAs of a tensor-core launch keep in step (advisory, all zero
+ *     between launches), and the scratch of a3po_loss_fwd_static.
  *   - Work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = legacy default
  *     stream).  Calls never synchronise the device and are asynchronous w.r.t. the host.
  *   - Return value: A3PO_OK or a negative a3po_error.  Argument errors are detected on the
