@@ -363,7 +363,11 @@ int a3po_train_step(const void* hidden, const int32_t* targets, const float* beh
  * end-to-end form of the call above):
  *   copies hidden, targets, behav_logp, versions, adv, mask host->device, runs a3po_train_step,
  *   copies loss + stats back.
- * h_* are host pointers (pinned memory recommended; pageable works but serialises).
+ * Of `hidden`, only the runs of rows with mask != 0 are copied when the step keeps its softmax
+ * (it reads no other row; the rest of the staged copy is then undefined); every row is copied
+ * when the workspace or the shape sends the step down the recomputing calls.
+ * h_* are host pointers (pinned memory recommended; pageable works but serialises); h_mask is
+ * read by the host during the call.
  * d_w, d_grad_w (accumulated into when accumulate_grad_w != 0), d_grad_hidden ([N,H] dt) and
  * d_stage/d_ws are device buffers.  d_stage needs a3po_train_step_stage_bytes(N,H,dt) bytes and
  * d_ws a3po_train_step_workspace_bytes(N,H,V,dt).  h_loss (float) and h_stats are host outputs,
@@ -378,6 +382,10 @@ int a3po_train_step_host(const void* h_hidden, const int32_t* h_targets, const f
                          int accumulate_grad_w, void* d_grad_hidden, void* d_stage,
                          size_t stage_bytes, void* d_ws, size_t ws_bytes, float* h_loss,
                          a3po_stats* h_stats, uint32_t* d_status, void* stream);
+
+/* Bytes the host entries of this library have copied host->device in the calling process since
+ * load (monotonic; for transfer accounting in benchmarks). */
+int64_t a3po_host_to_device_bytes(void);
 
 /* Number of kernels this library has launched in the calling process since load
  * (monotonic; for launch accounting in benchmarks). */

@@ -43,6 +43,7 @@ _SIGNATURES = {
     "a3po_token_logprobs_min_workspace_bytes": (c_size_t, [c_int64, c_int, c_int, c_int, c_int]),
     "a3po_loss_workspace_bytes": (c_size_t, [c_int64]),
     "a3po_train_step_stage_bytes": (c_size_t, [c_int64, c_int, c_int]),
+    "a3po_host_to_device_bytes": (c_int64, []),
     "a3po_train_step_workspace_bytes": (c_size_t, [c_int64, c_int, c_int, c_int]),
     "a3po_token_logprobs_fwd": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_int, c_int, c_int, c_float,
                                         c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p, c_void_p]),
@@ -179,6 +180,10 @@ def a3po_loss_workspace_bytes(N) -> int:
 
 def a3po_train_step_stage_bytes(N, H, dt) -> int:
     return load_library().a3po_train_step_stage_bytes(N, H, dt)
+
+
+def a3po_host_to_device_bytes() -> int:
+    return int(load_library().a3po_host_to_device_bytes())
 
 
 def a3po_train_step_workspace_bytes(N, H, V, dt) -> int:

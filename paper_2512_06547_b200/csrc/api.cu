@@ -1,7 +1,9 @@
 // C ABI of the LM-head log-prob calls, the whole-step host entry and library-wide helpers.
 
+#include <atomic>
 #include <cstring>
 #include <mutex>
+#include <utility>
 #include <vector>
 
 #include "a3po_common.cuh"
@@ -758,6 +760,43 @@ int a3po_train_step(const void* hidden, const int32_t* targets, const float* beh
   return loss_finalize_partials(partials, n_chunks * loss_blocks, loss, stats, stream);
 }
 
+namespace {
+
+// Runs [begin, end) of rows with mask != 0; two runs with fewer than min_gap rows between them are merged.
+// More than max_runs runs: one run from the first to the last such row.
+void mask_row_runs(const uint8_t* mask, long long n, long long min_gap, size_t max_runs,
+                   std::vector<std::pair<long long, long long>>* runs) {
+  runs->clear();
+  long long i = 0;
+  while (i < n) {
+    while (i < n && mask[i] == 0) {   // skip zeros, eight at a time where possible
+      if ((reinterpret_cast<uintptr_t>(mask + i) & 7u) == 0 && i + 8 <= n) {
+        uint64_t word;
+        std::memcpy(&word, mask + i, 8);
+        if (word == 0) { i += 8; continue; }
+      }
+      ++i;
+    }
+    if (i >= n) break;
+    const long long begin = i;
+    const void* z = std::memchr(mask + i, 0, static_cast<size_t>(n - i));
+    i = z ? static_cast<const uint8_t*>(z) - mask : n;
+    if (!runs->empty() && begin - runs->back().second < min_gap) runs->back().second = i;
+    else runs->emplace_back(begin, i);
+  }
+  if (runs->size() > max_runs) {
+    const long long first = runs->front().first, last = runs->back().second;
+    runs->clear();
+    runs->emplace_back(first, last);
+  }
+}
+
+std::atomic<long long> g_h2d_bytes{0};
+
+}  // namespace
+
+int64_t a3po_host_to_device_bytes(void) { return g_h2d_bytes.load(std::memory_order_relaxed); }
+
 int a3po_train_step_host(const void* h_hidden, const int32_t* h_targets, const float* h_behav_logp,
                          const int32_t* h_versions, const float* h_adv, const uint8_t* h_mask, int64_t N, int H,
                          int V, a3po_dtype dt, int32_t current_version, float clip_eps, float inv_temperature,
@@ -778,16 +817,38 @@ int a3po_train_step_host(const void* h_hidden, const int32_t* h_targets, const f
   auto h2d = [&](size_t off, const void* src, size_t bytes) -> bool {
     return bytes == 0 || cudaMemcpyAsync(base + off, src, bytes, cudaMemcpyHostToDevice, stream) == cudaSuccess;
   };
+  const void* hidden = base + s.hidden;
   {
     ProfileScope scope(kKH2D, stream);   // with the per-kernel profile on, the copies show up as one entry
-    if (!h2d(s.hidden, h_hidden, rows * H * elt_size(dt)) || !h2d(s.targets, h_targets, rows * 4) ||
-        !h2d(s.behav, h_behav_logp, rows * 4) || !h2d(s.versions, h_versions, rows * 4) ||
-        !h2d(s.adv, h_adv, rows * 4) || !h2d(s.mask, h_mask, rows)) {
+    bool ok = h2d(s.targets, h_targets, rows * 4) && h2d(s.behav, h_behav_logp, rows * 4) &&
+              h2d(s.versions, h_versions, rows * 4) && h2d(s.adv, h_adv, rows * 4) && h2d(s.mask, h_mask, rows);
+    size_t copied = rows * (4 + 4 + 4 + 4 + 1);
+    // The step that keeps the softmax reads `hidden` only at rows with mask != 0 (it gathers them by index), so
+    // only the runs of such rows cross the bus; runs closer together than a copy call is worth are merged.  The
+    // recomputing fallback may multiply masked rows as zero rows and therefore gets every row.
+    const size_t row_bytes = static_cast<size_t>(H) * elt_size(dt);
+    const bool kept_path = N > 0 && use_tc(dt, hidden, d_w, N, H, V) && aligned_to(d_grad_hidden, 16) &&
+                           aligned_to(d_grad_w, 16) && step_chunk_rows_for(ws_bytes, N, H, V) > 0;
+    if (kept_path) {
+      std::vector<std::pair<long long, long long>> runs;
+      const long long min_gap = static_cast<long long>((size_t(256) << 10) / row_bytes) + 1;
+      mask_row_runs(h_mask, N, min_gap, 1024, &runs);
+      for (const auto& r : runs) {
+        const size_t off = static_cast<size_t>(r.first) * row_bytes;
+        const size_t bytes = static_cast<size_t>(r.second - r.first) * row_bytes;
+        ok = ok && h2d(s.hidden + off, static_cast<const char*>(h_hidden) + off, bytes);
+        copied += bytes;
+      }
+    } else {
+      ok = ok && h2d(s.hidden, h_hidden, rows * row_bytes);
+      copied += rows * row_bytes;
+    }
+    if (!ok) {
       cudaGetLastError();
       return A3PO_ERR_CUDA;
     }
+    g_h2d_bytes.fetch_add(static_cast<long long>(copied), std::memory_order_relaxed);
   }
-  const void* hidden = base + s.hidden;
   const int32_t* targets = reinterpret_cast<const int32_t*>(base + s.targets);
   const float* behav = reinterpret_cast<const float*>(base + s.behav);
   const int32_t* versions = reinterpret_cast<const int32_t*>(base + s.versions);

@@ -64,17 +64,26 @@ def run_host_step(wl, behav):
     pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
     h_hidden = wl.hidden.cpu().pin_memory()
     stage = a3po.new_workspace(a3po.a3po_train_step_stage_bytes(wl.N, wl.H, dt))
+    stage.fill_(0xFF)       # rows of hidden that are not copied (mask 0) read as NaN: nothing may depend on them
     ws = a3po.new_workspace(a3po.a3po_train_step_workspace_bytes(wl.N, wl.H, wl.V, dt))
     grad_w = torch.zeros((wl.V, wl.H), dtype=torch.float32, device=DEV)
     grad_hidden = torch.empty_like(wl.hidden)
     h_loss = torch.zeros(1).pin_memory()
     h_stats = torch.zeros(24, dtype=torch.uint8).pin_memory()
     status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    copied = a3po.a3po_host_to_device_bytes()
     a3po.a3po_train_step_host(h_hidden, pin(wl.targets), pin(behav), pin(wl.versions), pin(wl.adv), pin(wl.mask),
                               wl.current_version, wl.clip_eps, wl.w, grad_w, grad_hidden, stage, ws, h_loss,
                               h_stats=h_stats, d_status=status)
     torch.cuda.synchronize()
     assert int(status.item()) == 0
+    # transfer accounting: the per-token arrays in full, of hidden at least the rows that take part, at most all
+    copied = a3po.a3po_host_to_device_bytes() - copied
+    row_bytes = wl.H * h_hidden.element_size()
+    small = wl.N * (4 + 4 + 4 + 4 + 1)
+    assert small + int((wl.mask != 0).sum()) * row_bytes <= copied <= small + wl.N * row_bytes
+    if wl.dtype == "bf16" and wl.meta["recipe"].get("packed") is False:
+        assert copied < small + wl.N * row_bytes          # right padding stays on the host
     return float(h_loss.item()), a3po.read_stats(h_stats), grad_hidden, grad_w
 
 
