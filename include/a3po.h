@@ -15,6 +15,10 @@
  *     between launches), and the scratch of a3po_loss_fwd_static.
  *   - Work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = legacy default
  *     stream).  Calls never synchronise the device and are asynchronous w.r.t. the host.
+ *     A call with device inputs is a fixed sequence of launches (row counts stay on the
+ *     device), so it may be captured into a CUDA graph and replayed; make one uncaptured call
+ *     per device first (it resolves kernel attributes and the addresses of the library's
+ *     device arrays).
  *   - Return value: A3PO_OK or a negative a3po_error.  Argument errors are detected on the
  *     host before anything is launched; nothing is written in that case.
  *   - Conditions that only the device can see (a target index outside [0,V), a bounded wait

@@ -231,3 +231,45 @@ def test_loss_scale_and_data_parallel_helpers(ws_kind):
     assert float(res["scale"].item()) == 1.0 and int(res["m_global"].item()) == int(wl.mask.sum())
     assert float(res["loss"].item()) == pytest.approx(float(plain["loss"].item()), rel=1e-6)
     assert torch.equal(res["grad_w"], plain["grad_w"]) and torch.equal(res["grad_logp"], plain["grad_logp"])
+
+
+def test_step_replays_from_a_cuda_graph():
+    """The whole step is a fixed sequence of launches on one stream (row counts stay on the device), so it can be
+    captured once and replayed: same bits as the eager call, for new input values in the same buffers too."""
+    wl = make("1p5b", dict(V=8192 + 24, n_prompts=2, group=4, row_len=200, len_lo=30, len_hi=200), True)
+    ref = oracle_step(wl, wl.hidden, wl.w)
+    dt = a3po.A3PO_BF16
+    ws_bytes = a3po.a3po_train_step_workspace_bytes(wl.N, wl.H, wl.V, dt)
+    eager = _device_step(wl, ref["behav"], ws_bytes)              # also the uncaptured first call on this device
+    to_dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(DEV)
+    n = wl.N
+    targets, behav, versions, adv, mask = (to_dev(x) for x in (wl.targets, ref["behav"], wl.versions, wl.adv, wl.mask))
+    out = dict(logp=torch.empty(n, device=DEV), lse=torch.empty(n, device=DEV), grad_logp=torch.empty(n, device=DEV),
+               loss=torch.zeros(1, device=DEV), grad_hidden=torch.empty_like(wl.hidden),
+               grad_w=torch.empty((wl.V, wl.H), dtype=torch.float32, device=DEV), entropy=torch.empty(n, device=DEV))
+    stats = a3po.new_stats()
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    ws = a3po.new_workspace(ws_bytes)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        a3po.a3po_train_step(wl.hidden, wl.w, targets, behav, versions, wl.current_version, adv, mask, wl.clip_eps,
+                             out["logp"], out["lse"], out["grad_logp"], out["loss"], out["grad_hidden"], out["grad_w"],
+                             ws, stats=stats, entropy=out["entropy"], status=status)
+    for _ in range(2):
+        for t in out.values():
+            t.fill_(7.0)
+        graph.replay()
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        for k, t in out.items():
+            assert torch.equal(t, eager[k]), k
+    # other inputs in the same buffers: half of the tokens masked out, the replay follows the device-side counts
+    mask2 = wl.mask.copy()
+    mask2[::2] = 0
+    mask.copy_(to_dev(mask2))
+    graph.replay()
+    torch.cuda.synchronize()
+    wl.mask = mask2
+    eager2 = _device_step(wl, ref["behav"], ws_bytes)
+    for k, t in out.items():
+        assert torch.equal(t, eager2[k]), k
