@@ -515,7 +515,10 @@ def run_ours(args):
                    "H": h, "V": v, "parallelism": f"dp{world} (independent shards)",
                    "workspace_gib": round(r["ws_bytes"] / 2 ** 30, 2),
                    "l2": "no flush: W (%.0f MB) and the kept-probabilities scratch are larger than the 126 MB L2"
-                         % (v * h * 2 / 1e6)},
+                         % (v * h * 2 / 1e6),
+                   **({"library": "tuning build: " + (" ".join(f"{k}={val}" for k, val in sorted(os.environ.items())
+                                                               if k.startswith("A3PO_")) or "no switches set")}
+                      if args.library == "tuning" else {})},
         "rows_per_s": total_rows * args.steps / (ms_total * 1e-3),
         "executed_tflops": round(step_flops * world / (ms_per_step * 1e-3) / 1e12, 1),
         "rows_processed": {"fwd": n_valid, "bwd": r["bwd_rows"], "of": n},
@@ -687,7 +690,13 @@ def main():
     ap.add_argument("--separate-calls", action="store_true",
                     help="time fwd / loss / bwd as three ABI calls (backward recomputes the logits) instead of "
                          "a3po_train_step")
+    ap.add_argument("--library", default="product", choices=["product", "tuning"],
+                    help="tuning: load lib/liba3po_tuning.so (same sources, -DA3PO_TUNING), whose scheduling constants "
+                         "follow the A3PO_* environment variables; for A/B runs, not a benchmark number")
     args = ap.parse_args()
+    if args.library == "tuning":
+        from paper_2512_06547_b200 import binding, build as a3po_build
+        binding.LIB_PATH = a3po_build.build(tuning=True)
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
         sys.exit(respawn_under_torchrun(args))
     if args.workload == "loss_sweep":

@@ -52,7 +52,8 @@ int scatter_rows(const void* src_c, int h, const int* pos, long long n, void* ds
 
 // ---- tcgen05 / TMEM / TMA kernels (lmhead_tc.cu), bf16 only ----
 bool lmhead_tc_supported(const void* hidden, const void* w, long long n, int h, int v);
-// Vocabulary splits the tensor-core forward wants for (n, v): each (row tile, split) pair is one work item.
+// Vocabulary splits the tensor-core forward wants for n rows of h, v columns: each (row tile, split) pair is one
+// work item.
 int lmhead_tc_fwd_splits(long long n, int h, int v);
 // `dyn_rows` (device, may be null): number of rows of `hidden` that are really present (compact row space);
 // partials are laid out [split][n] regardless.
