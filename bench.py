@@ -674,7 +674,7 @@ def respawn_under_torchrun(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=12)   # 8B-shaped: 12 x 0.2 s, a timed region above LONG_REGION_S
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="8b", choices=sorted(WORKLOAD_TEXT) + ["loss_sweep"])
