@@ -47,6 +47,10 @@ METRIC = "logprob+A-3PO loss fwd/bwd tokens/s; % of bf16 TC peak & HBM roofline"
 NCU_TRAFFIC_PER_STEP = {
     "8b": {"gemm_tn<fwd_logsoftmax+keep>": 21.48e9 + 19.90e9 + 5.90e9 + 4.43e9},
     "1p5b": {"gemm_tn<fwd_logsoftmax+keep>": 0.70e9 + 2.72e9},
+    # not captured (the step holds 60 GB and runs 2.6 s): the same kernel on the same 65,536-row chunks as the 8B-shaped
+    # capture, whose traffic is per chunk launch; 16 full chunks plus one of 8,207 rows scaled by rows from the
+    # 14,545-row launch
+    "8b_packed": {"gemm_tn<fwd_logsoftmax+keep>": 16 * (21.48e9 + 19.90e9) + (5.90e9 + 4.43e9) * 8207 / 14545},
 }
 # Fused loss kernel (profiles/loss_kernel_16Mi_tokens_ncu_full.md): DRAM bytes per token at N = 2^24 (17 B read exactly;
 # most of the 4 B of gradient written per token is still in L2 when the kernel ends).
