@@ -685,7 +685,8 @@ def main():
     ap.add_argument("--tokens", type=int, default=1 << 26, help="token count of --workload loss_sweep")
     ap.add_argument("--min-seconds", type=float, default=1.5,
                     help="length of the timed window of --workload loss_sweep (short values for profiler captures)")
-    ap.add_argument("--oracle-rows", type=int, default=256)
+    ap.add_argument("--oracle-rows", type=int, default=1024,
+                    help="valid rows of the batch the CPU oracle is timed on (about 12 s on 16 cores at the 8B shape)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-configs", action="store_true",
                     help="skip the compact entries for the other named configurations")
