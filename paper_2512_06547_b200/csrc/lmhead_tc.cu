@@ -1165,8 +1165,11 @@ int launch_gemm(const Operand& a, const Operand& b, int splits, const typename E
   im.n_tiles = static_cast<int>((b.mn_extent + BN - 1) / BN);
   im.splits = splits > 0 ? splits : im.n_tiles;
   im.items = static_cast<long long>(im.m_tiles) * im.splits;
+  // hidden x W^T with one tile per item (the recomputed dz) sweeps W like the forward does
+  constexpr bool kForwardLike = !A_MN && !B_MN;
   im.group_m = splits > 0 ? tuning_override("A3PO_GROUP_M", fwd_group_m(a.k_extent))
-                          : tuning_override("A3PO_GROUP_M_GRAD", kGroupM);
+               : kForwardLike ? tuning_override("A3PO_GROUP_M_DZ", fwd_group_m(a.k_extent))
+                              : tuning_override("A3PO_GROUP_M_GRAD", kGroupM);
   im.dyn_rows = dyn.rows;
   im.dyn_is_k = dyn.is_k;
   im.zero_when_empty = dyn.zero_when_empty;
